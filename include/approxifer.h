@@ -1,0 +1,155 @@
+/*
+ * approxifer.h  --  C ABI of the ApproxIFER encode / decode / locate library for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel hot path of ApproxIFER
+ * (arXiv 2109.09868, Section 3): the Berrut rational-interpolation encoder,
+ * the straggler-masked Berrut decoder and the Byzantine-worker locator
+ * (Algorithm 2), over G independent groups at a time.
+ *
+ * Notation.  K = queries per group (j = 0..K-1).  W = number of workers =
+ * number of coded queries (i = 0..W-1); the paper counts workers 0..N, so
+ * W = N+1.  E = Byzantine workers to locate.  D / C = payload elements per
+ * query / per prediction.  Nodes (Section 3, "Encoding"):
+ *     alpha_j = cos((2j+1) pi / (2K)),      beta_i = cos(i pi / (W-1)).
+ *
+ * Common rules for every entry point
+ *   - All array arguments are DEVICE pointers owned by the caller (global
+ *     memory of the current device), fp32 payloads, innermost dimension
+ *     contiguous; "gstride" / "rstride" are the distances, in ELEMENTS, between
+ *     consecutive groups / consecutive rows of a group.  Inputs and outputs
+ *     must not overlap.  `params` is a HOST pointer, read during the call.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL =
+ *     the legacy default stream) and the call returns without synchronising.
+ *     The library allocates no memory, keeps no per-call state and may be
+ *     called from several host threads on different streams.
+ *   - 16-byte aligned bases with D (or C) and all strides multiples of 4 take
+ *     the 128-bit fast path; anything else runs a slower element-wise GPU
+ *     path.  There is no CPU fallback.
+ *   - Return value: APPROXIFER_OK or a negative APPROXIFER_E_* code.  Argument
+ *     errors are detected on the host before anything is launched.  G == 0 is
+ *     a valid no-op.
+ *   - Per-group conditions are reported as APPROXIFER_ST_* bits in the
+ *     optional `status[G]` output, never as a fault.
+ */
+#ifndef APPROXIFER_H_
+#define APPROXIFER_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define APPROXIFER_VERSION 100 /* major*10000 + minor*100 + patch */
+
+#define APPROXIFER_MAX_K 32
+#define APPROXIFER_MAX_W 32
+
+/* return codes */
+#define APPROXIFER_OK 0
+#define APPROXIFER_E_NULL (-1)  /* a required pointer is NULL */
+#define APPROXIFER_E_RANGE (-2) /* K not in 1..32, W not in 2..32, E < 0, G < 0, D < 1, D > 2^31, stride < row length */
+#define APPROXIFER_E_PARAM (-3) /* locate: E < 1 or 2(K+E) > W; unknown flag bits */
+#define APPROXIFER_E_CUDA (-4)  /* the CUDA runtime reported an error at launch */
+
+/* params.flags */
+#define APPROXIFER_SIGN_RANK 0u         /* decoder sign (-1)^(rank of worker i among those used); default */
+#define APPROXIFER_SIGN_WORKER_INDEX 1u /* decoder sign (-1)^i, the decoding equation read literally */
+
+/* status[g] bits */
+#define APPROXIFER_ST_NO_WORKERS 1u             /* decode: no worker present; the group's output is zero-filled */
+#define APPROXIFER_ST_FEW_WORKERS 2u            /* decode: fewer than K workers present; computed anyway */
+#define APPROXIFER_ST_LOCATE_UNDERDETERMINED 4u /* locate: fewer than 2(K+E) workers present; nothing located */
+#define APPROXIFER_ST_NONFINITE 8u              /* locate: some Q(beta_i) was not finite (ranked as +inf) */
+
+typedef struct approxifer_params {
+  int32_t K;      /* 1..32 queries per group */
+  int32_t W;      /* 2..32 workers (paper: N+1) */
+  int32_t E;      /* Byzantine workers to locate; ignored by encode and decode */
+  uint32_t flags; /* APPROXIFER_SIGN_* */
+} approxifer_params;
+
+/*
+ * Encoder (Section 3, "ApproxIFER Encoding"):
+ *     Xt[g][i][:] = u_g(beta_i) = sum_j l_j(beta_i) X[g][j][:],
+ *     l_j(z) = [(-1)^j/(z-alpha_j)] / sum_k (-1)^k/(z-alpha_k).
+ * If beta_i equals some alpha_j (exactly when (2j+1)(W-1) == 2Ki) the row is
+ * the limit value X[g][j][:].
+ *   X   in,  [G][K][D], strides x_gstride >= ?, x_rstride >= D (elements)
+ *   Xt  out, [G][W][D], strides xt_gstride, xt_rstride >= D; a worker-major
+ *            layout [W][G][D] is expressed as xt_gstride = D, xt_rstride = G*D.
+ * fp32 accumulation, one fused multiply-add per term, j ascending.
+ */
+int approxifer_encode(const approxifer_params* params, int64_t G, int64_t D,
+                      const float* X, int64_t x_gstride, int64_t x_rstride,
+                      float* Xt, int64_t xt_gstride, int64_t xt_rstride,
+                      void* cuda_stream);
+
+/*
+ * Decoder (Section 3, "ApproxIFER Decoding", step 2):
+ *     Yhat[g][j][:] = r_g(alpha_j),
+ *     r_g(z) = sum_{i in F_g} [s_i/(z-beta_i)] Yt[g][i][:] / sum_{i in F_g} s_i/(z-beta_i),
+ * F_g = workers whose bit is set in mask[g] (bits >= W are ignored), taken in
+ * ascending order; s_i = (-1)^(position of i in F_g) by default, (-1)^i with
+ * APPROXIFER_SIGN_WORKER_INDEX.  Every worker in the mask is used.  If
+ * alpha_j equals beta_i for a present worker i, Yhat[g][j][:] = Yt[g][i][:].
+ *   Yt      in,  [G][W][C]; rows of absent workers may hold anything (NaN
+ *                included) and never influence the output
+ *   mask    in,  [G] uint32, bit i = worker i's prediction arrived
+ *   Yhat    out, [G][K][C]
+ *   n_used  out, [G] int32 = |F_g|, or NULL
+ *   status  out, [G] uint32 of APPROXIFER_ST_* bits, or NULL
+ */
+int approxifer_decode(const approxifer_params* params, int64_t G, int64_t C,
+                      const float* Yt, int64_t yt_gstride, int64_t yt_rstride,
+                      const uint32_t* mask,
+                      float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                      int32_t* n_used, uint32_t* status, void* cuda_stream);
+
+/*
+ * Byzantine-worker locator (Algorithm 2; Algorithm 1 is its inner step; the
+ * theory is Appendix A, Theorem 1).  For every group and every class c:
+ * least-squares solution of
+ *     P(beta_i) = Yt[g][i][c] * Q(beta_i),   i in A_avl (the mask),
+ *     P(x) = sum_{k<K+E} P_k x^k,  Q(x) = 1 + sum_{1<=k<K+E} Q_k x^k,
+ * a_i = Q(beta_i), the E workers with the smallest |a_i| get one vote each;
+ * the E workers with the most votes over all classes are reported.  Ties, in
+ * both selections, go to the lower worker index.  The solve runs in fp64.
+ *   adv           out, [G][E] int32, ascending; -1 when nothing was located
+ *   trusted_mask  out, [G] uint32 = mask (bits < W) minus the located workers
+ *   status        out, [G] uint32 or NULL
+ * Requires E >= 1 and 2(K+E) <= W.  A group with fewer than 2(K+E) workers
+ * present gets adv = -1, trusted_mask = mask and ST_LOCATE_UNDERDETERMINED.
+ */
+int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C,
+                      const float* Yt, int64_t yt_gstride, int64_t yt_rstride,
+                      const uint32_t* mask,
+                      int32_t* adv, uint32_t* trusted_mask, uint32_t* status,
+                      void* cuda_stream);
+
+/*
+ * Test hook (not on the hot path): the weights the kernels use, computed on
+ * the device by the same code.
+ *   which = 0: encoder, w[W][K] = l_j(beta_i);            idx, n untouched
+ *   which = 1: decoder for one `mask`, w[K][W] with columns 0..n-1 holding the
+ *              weights of the n workers used (rest 0), idx[W] their indices
+ *              (rest -1), *n their number (Section 3, decoding).
+ * w, idx, n are device pointers.
+ */
+int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int which,
+                             float* w, int32_t* idx, int32_t* n, void* cuda_stream);
+
+/* Human-readable text for a return code (static storage). */
+const char* approxifer_strerror(int code);
+
+/* APPROXIFER_VERSION of the loaded library. */
+int approxifer_version(void);
+
+/* Number of kernels this library has launched in this process so far. */
+int64_t approxifer_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* APPROXIFER_H_ */

@@ -1,0 +1,22 @@
+"""ApproxIFER encode / decode / locate for NVIDIA B200 (sm_100a).
+
+The product is the C-ABI shared library ``libapproxifer.so`` (declared in
+``include/approxifer.h``, sources in ``csrc/``); this package is its thin
+Python binding plus the seeded workload generators used by the tests and the
+benchmark.
+"""
+from .binding import (  # noqa: F401
+    ApproxiferError,
+    approxifer_debug_weights,
+    approxifer_decode,
+    approxifer_encode,
+    approxifer_locate,
+    approxifer_params,
+    launch_count,
+    library_path,
+    load,
+    make_params,
+    mask_tensor,
+    strerror,
+    version,
+)

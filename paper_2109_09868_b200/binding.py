@@ -1,0 +1,205 @@
+"""Thin Python binding of ``libapproxifer.so`` (declared in ``include/approxifer.h``).
+
+Argument marshalling only: tensors are turned into device pointers and element
+strides, and the C entry point of the same name is called.  Every step of the
+computation runs in the library's CUDA kernels; there is no fallback of any
+kind -- a missing library or a non-CUDA tensor raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import shutil
+from ctypes import POINTER, c_char_p, c_float, c_int, c_int32, c_int64, c_uint32, c_void_p
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+OK = 0
+E_NULL, E_RANGE, E_PARAM, E_CUDA = -1, -2, -3, -4
+SIGN_RANK, SIGN_WORKER_INDEX = 0, 1
+ST_NO_WORKERS, ST_FEW_WORKERS, ST_LOCATE_UNDERDETERMINED, ST_NONFINITE = 1, 2, 4, 8
+
+EXPORTS = (
+    "approxifer_encode",
+    "approxifer_decode",
+    "approxifer_locate",
+    "approxifer_debug_weights",
+    "approxifer_strerror",
+    "approxifer_version",
+    "approxifer_launch_count",
+)
+
+
+class approxifer_params(ctypes.Structure):
+    _fields_ = [("K", c_int32), ("W", c_int32), ("E", c_int32), ("flags", c_uint32)]
+
+
+class ApproxiferError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: %s (code %d)" % (where, strerror(code), code))
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load() -> ctypes.CDLL:
+    """Load the CUDA library, (re)building it first if nvcc is present and the
+    sources are newer.  Raises if no library can be had."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    have_nvcc = shutil.which("nvcc") is not None or os.path.exists("/usr/local/cuda/bin/nvcc")
+    if have_nvcc and _build.is_stale():
+        _build.build()
+    if not os.path.exists(_build.LIB):
+        raise RuntimeError(
+            "libapproxifer.so is missing and cannot be built (no nvcc): run `python -m paper_2109_09868_b200.build`"
+        )
+    lib = ctypes.CDLL(_build.LIB)
+    pf, pu, pi = POINTER(c_float), POINTER(c_uint32), POINTER(c_int32)
+    pp = POINTER(approxifer_params)
+    lib.approxifer_encode.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p]
+    lib.approxifer_encode.restype = c_int
+    lib.approxifer_decode.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_int64,
+                                      c_int64, c_void_p, c_void_p, c_void_p]
+    lib.approxifer_decode.restype = c_int
+    lib.approxifer_locate.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
+                                      c_void_p, c_void_p]
+    lib.approxifer_locate.restype = c_int
+    lib.approxifer_debug_weights.argtypes = [pp, c_uint32, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.approxifer_debug_weights.restype = c_int
+    lib.approxifer_strerror.argtypes = [c_int]
+    lib.approxifer_strerror.restype = c_char_p
+    lib.approxifer_version.restype = c_int
+    lib.approxifer_launch_count.restype = c_int64
+    del pf, pu, pi
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().approxifer_strerror(int(code)).decode()
+
+
+def version() -> int:
+    return int(load().approxifer_version())
+
+
+def launch_count() -> int:
+    return int(load().approxifer_launch_count())
+
+
+def make_params(K: int, W: int, E: int = 0, flags: int = 0) -> approxifer_params:
+    return approxifer_params(int(K), int(W), int(E), int(flags))
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _payload(t: torch.Tensor, rows: int, name: str):
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor (the library has no CPU path)" % name)
+    if t.dtype != torch.float32 or t.dim() != 3 or t.shape[1] != rows:
+        raise ValueError("%s must be float32 [G][%d][L]" % (name, rows))
+    if t.shape[2] > 1 and t.stride(2) != 1:
+        raise ValueError("%s: innermost dimension must be contiguous" % name)
+    return t.data_ptr(), t.stride(0), t.stride(1)
+
+
+def _vec(t: Optional[torch.Tensor], dtype, n: int, name: str) -> int:
+    if t is None:
+        return 0
+    if not t.is_cuda or t.dtype != dtype or t.numel() != n or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous CUDA %s tensor with %d elements" % (name, dtype, n))
+    return t.data_ptr()
+
+
+def approxifer_encode(params: approxifer_params, X: torch.Tensor, Xt: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """X [G][K][D] -> coded queries Xt [G][W][D] (allocated if not given)."""
+    G, K, D = X.shape
+    if Xt is None:
+        Xt = torch.empty((G, params.W, D), device=X.device, dtype=torch.float32)
+    xp, xg, xr = _payload(X, params.K, "X")
+    op, og, orr = _payload(Xt, params.W, "Xt")
+    if Xt.shape[0] != G or Xt.shape[2] != D:
+        raise ValueError("Xt must be [G][W][D]")
+    rc = load().approxifer_encode(ctypes.byref(params), G, D, xp, xg, xr, op, og, orr, _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_encode")
+    return Xt
+
+
+def approxifer_decode(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, Yhat: Optional[torch.Tensor] = None,
+                      n_used: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Yt [G][W][C], mask [G] (int32 tensor holding the uint32 bit patterns) -> Yhat [G][K][C]."""
+    G, W, C = Yt.shape
+    if Yhat is None:
+        Yhat = torch.empty((G, params.K, C), device=Yt.device, dtype=torch.float32)
+    yp, yg, yr = _payload(Yt, params.W, "Yt")
+    op, og, orr = _payload(Yhat, params.K, "Yhat")
+    if Yhat.shape[0] != G or Yhat.shape[2] != C:
+        raise ValueError("Yhat must be [G][K][C]")
+    mp = _vec(mask, torch.int32, G, "mask")
+    rc = load().approxifer_decode(ctypes.byref(params), G, C, yp, yg, yr, mp, op, og, orr,
+                                  _vec(n_used, torch.int32, G, "n_used"), _vec(status, torch.int32, G, "status"),
+                                  _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_decode")
+    return Yhat
+
+
+def approxifer_locate(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, adv: Optional[torch.Tensor] = None,
+                      trusted_mask: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, stream=None):
+    """Yt [G][W][C], mask [G] -> (adv [G][E] int32, trusted_mask [G] int32 bit patterns)."""
+    G, W, C = Yt.shape
+    E = max(int(params.E), 0)
+    if adv is None:
+        adv = torch.empty((G, E), device=Yt.device, dtype=torch.int32)
+    if trusted_mask is None:
+        trusted_mask = torch.empty((G,), device=Yt.device, dtype=torch.int32)
+    yp, yg, yr = _payload(Yt, params.W, "Yt")
+    rc = load().approxifer_locate(ctypes.byref(params), G, C, yp, yg, yr, _vec(mask, torch.int32, G, "mask"),
+                                  _vec(adv, torch.int32, G * E, "adv"), _vec(trusted_mask, torch.int32, G, "trusted_mask"),
+                                  _vec(status, torch.int32, G, "status"), _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_locate")
+    return adv, trusted_mask
+
+
+def approxifer_debug_weights(params: approxifer_params, mask: int = 0, which: int = 0, stream=None):
+    """which=0: encoder weights [W][K]; which=1: (decoder weights [K][n], worker indices) for `mask`."""
+    dev = torch.device("cuda")
+    K, W = params.K, params.W
+    if which == 0:
+        w = torch.empty((W, K), device=dev, dtype=torch.float32)
+        rc = load().approxifer_debug_weights(ctypes.byref(params), 0, 0, w.data_ptr(), 0, 0, _stream_ptr(stream))
+        if rc != OK:
+            raise ApproxiferError(rc, "approxifer_debug_weights")
+        return w
+    w = torch.empty((K, W), device=dev, dtype=torch.float32)
+    idx = torch.empty((W,), device=dev, dtype=torch.int32)
+    n = torch.empty((1,), device=dev, dtype=torch.int32)
+    rc = load().approxifer_debug_weights(ctypes.byref(params), int(mask) & 0xFFFFFFFF, 1, w.data_ptr(), idx.data_ptr(),
+                                         n.data_ptr(), _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_debug_weights")
+    nn = int(n.item())
+    return w[:, :nn], idx[:nn]
+
+
+def mask_tensor(mask_u32, device="cuda") -> torch.Tensor:
+    """numpy uint32 [G] -> int32 tensor with the same bit patterns on `device`."""
+    import numpy as np
+
+    return torch.from_numpy(np.ascontiguousarray(mask_u32, dtype=np.uint32).view(np.int32).copy()).to(device)

@@ -1,0 +1,109 @@
+// C ABI of the ApproxIFER library: argument validation and dispatch.
+// The declarations and their contracts are in include/approxifer.h.
+#include <atomic>
+
+#include "../../include/approxifer.h"
+#include "common.cuh"
+
+namespace approxifer {
+
+namespace {
+std::atomic<long long> g_launches{0};
+}
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+namespace {
+
+int check_kw(const approxifer_params* p) {
+  if (p == nullptr) return APPROXIFER_E_NULL;
+  if (p->K < 1 || p->K > APPROXIFER_MAX_K || p->W < 2 || p->W > APPROXIFER_MAX_W) return APPROXIFER_E_RANGE;
+  if (p->flags & ~APPROXIFER_SIGN_WORKER_INDEX) return APPROXIFER_E_PARAM;
+  return APPROXIFER_OK;
+}
+
+// [G][rows][len] with element strides gs, rs: rows must not overlap.
+int check_layout(int64_t G, int64_t len, int64_t rs) {
+  if (G < 0 || len < 1 || len > (int64_t(1) << 31)) return APPROXIFER_E_RANGE;
+  if (rs < len) return APPROXIFER_E_RANGE;
+  return APPROXIFER_OK;
+}
+
+int from_cuda(cudaError_t e) { return e == cudaSuccess ? APPROXIFER_OK : APPROXIFER_E_CUDA; }
+
+}  // namespace
+}  // namespace approxifer
+
+using namespace approxifer;
+
+extern "C" {
+
+int approxifer_encode(const approxifer_params* params, int64_t G, int64_t D, const float* X, int64_t x_gstride,
+                      int64_t x_rstride, float* Xt, int64_t xt_gstride, int64_t xt_rstride, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if ((rc = check_layout(G, D, x_rstride))) return rc;
+  if ((rc = check_layout(G, D, xt_rstride))) return rc;
+  if (x_gstride < 0 || xt_gstride < 0) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (X == nullptr || Xt == nullptr) return APPROXIFER_E_NULL;
+  EncodeArgs a{X, Xt, x_gstride, x_rstride, xt_gstride, xt_rstride, G, D, params->K, params->W};
+  return from_cuda(launch_encode(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int approxifer_decode(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
+                      int64_t yt_rstride, const uint32_t* mask, float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                      int32_t* n_used, uint32_t* status, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if ((rc = check_layout(G, C, yt_rstride))) return rc;
+  if ((rc = check_layout(G, C, yh_rstride))) return rc;
+  if (yt_gstride < 0 || yh_gstride < 0) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (Yt == nullptr || Yhat == nullptr || mask == nullptr) return APPROXIFER_E_NULL;
+  DecodeArgs a{Yt,         mask,       Yhat,       n_used, status, yt_gstride, yt_rstride,
+               yh_gstride, yh_rstride, G,          C,      params->K, params->W, params->flags};
+  return from_cuda(launch_decode(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
+                      int64_t yt_rstride, const uint32_t* mask, int32_t* adv, uint32_t* trusted_mask, uint32_t* status,
+                      void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if (params->E < 0) return APPROXIFER_E_RANGE;
+  if (params->E < 1 || 2 * (params->K + params->E) > params->W) return APPROXIFER_E_PARAM;
+  if ((rc = check_layout(G, C, yt_rstride))) return rc;
+  if (yt_gstride < 0) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (Yt == nullptr || mask == nullptr || adv == nullptr || trusted_mask == nullptr) return APPROXIFER_E_NULL;
+  LocateArgs a{Yt, mask, adv, trusted_mask, status, yt_gstride, yt_rstride, G, C, params->K, params->W, params->E};
+  return from_cuda(launch_locate(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int which, float* w, int32_t* idx,
+                             int32_t* n, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if (which != 0 && which != 1) return APPROXIFER_E_PARAM;
+  if (w == nullptr || (which == 1 && (idx == nullptr || n == nullptr))) return APPROXIFER_E_NULL;
+  return from_cuda(launch_debug_weights(params->K, params->W, params->flags, mask, which, w, idx, n,
+                                        static_cast<cudaStream_t>(cuda_stream)));
+}
+
+const char* approxifer_strerror(int code) {
+  switch (code) {
+    case APPROXIFER_OK: return "ok";
+    case APPROXIFER_E_NULL: return "a required pointer is NULL";
+    case APPROXIFER_E_RANGE: return "argument out of range (K in 1..32, W in 2..32, E >= 0, G >= 0, 1 <= D <= 2^31, row stride >= row length)";
+    case APPROXIFER_E_PARAM: return "inconsistent parameters (locate needs E >= 1 and 2(K+E) <= W; unknown flag bits)";
+    case APPROXIFER_E_CUDA: return "the CUDA runtime reported an error at kernel launch";
+    default: return "unknown error code";
+  }
+}
+
+int approxifer_version(void) { return APPROXIFER_VERSION; }
+
+int64_t approxifer_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

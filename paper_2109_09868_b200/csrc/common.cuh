@@ -1,0 +1,72 @@
+// Shared declarations of the ApproxIFER CUDA library (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "tables.h"
+
+namespace approxifer {
+
+// status[g] bits (mirrors approxifer.h)
+constexpr uint32_t kStNoWorkers = 1u;
+constexpr uint32_t kStFewWorkers = 2u;
+constexpr uint32_t kStLocateUnderdetermined = 4u;
+constexpr uint32_t kStNonfinite = 8u;
+
+constexpr uint32_t kFlagSignWorkerIndex = 1u;
+
+struct EncodeArgs {
+  const float* X;
+  float* Xt;
+  int64_t x_gs, x_rs, o_gs, o_rs;  // element strides
+  int64_t G, D;
+  int32_t K, W;
+};
+
+struct DecodeArgs {
+  const float* Yt;
+  const uint32_t* mask;
+  float* Yh;
+  int32_t* n_used;
+  uint32_t* status;
+  int64_t y_gs, y_rs, o_gs, o_rs;
+  int64_t G, C;
+  int32_t K, W;
+  uint32_t flags;
+};
+
+struct LocateArgs {
+  const float* Yt;
+  const uint32_t* mask;
+  int32_t* adv;
+  uint32_t* trusted;
+  uint32_t* status;
+  int64_t y_gs, y_rs;
+  int64_t G, C;
+  int32_t K, W, E;
+};
+
+// Each returns a cudaError_t from the launch (cudaSuccess if nothing to do).
+cudaError_t launch_encode(const EncodeArgs& a, cudaStream_t stream);
+cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
+cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream);
+cudaError_t launch_debug_weights(int K, int W, uint32_t flags, uint32_t mask, int which, float* w, int32_t* idx,
+                                 int32_t* n, cudaStream_t stream);
+
+void count_launch(int n = 1);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+#ifdef __CUDACC__
+// Streaming (evict-first) 128-bit and 32-bit global accesses: every payload
+// byte is touched exactly once.
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+__device__ __forceinline__ float ld_stream(const float* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
+__device__ __forceinline__ void st_stream(float* p, float v) { __stcs(p, v); }
+
+__device__ __forceinline__ uint32_t worker_bits(int W) { return W >= 32 ? 0xffffffffu : ((1u << W) - 1u); }
+#endif
+
+}  // namespace approxifer

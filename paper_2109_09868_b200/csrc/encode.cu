@@ -1,0 +1,101 @@
+// ApproxIFER encoder kernels (Section 3, "Encoding"):
+//   Xt[g][i][:] = sum_j l_j(beta_i) X[g][j][:]
+// A skinny (W x K) weighted sum per payload column: HBM-bound, no reuse beyond
+// registers.  Each thread owns one 16-byte (or, on the unaligned path, 4-byte)
+// column of one group: it loads its K inputs with streaming loads, then forms
+// the W output rows one after another and streams them out.  The weights are
+// launch constants living in the kernel-parameter constant bank.
+#include "common.cuh"
+
+namespace approxifer {
+
+namespace {
+
+constexpr int kEncodeThreads = 256;
+
+template <typename V>
+struct VecOps;
+template <>
+struct VecOps<float4> {
+  static constexpr int kLanes = 4;
+  static __device__ __forceinline__ float4 mul(float w, float4 x) { return make_float4(w * x.x, w * x.y, w * x.z, w * x.w); }
+  static __device__ __forceinline__ float4 fma(float w, float4 x, float4 a) {
+    return make_float4(fmaf(w, x.x, a.x), fmaf(w, x.y, a.y), fmaf(w, x.z, a.z), fmaf(w, x.w, a.w));
+  }
+};
+template <>
+struct VecOps<float> {
+  static constexpr int kLanes = 1;
+  static __device__ __forceinline__ float mul(float w, float x) { return w * x; }
+  static __device__ __forceinline__ float fma(float w, float x, float a) { return fmaf(w, x, a); }
+};
+
+// One work item = (group g, column v) with v counting V-wide columns of the
+// payload; items are numbered g*Dv + v and dealt to threads in order, so a
+// warp reads and writes 32 consecutive columns of a row.
+template <int K, typename V>
+__global__ void __launch_bounds__(kEncodeThreads) encode_kernel(const __grid_constant__ EncodeArgs a,
+                                                                const __grid_constant__ EncodeTables tab) {
+  using Ops = VecOps<V>;
+  const uint32_t Dv = (uint32_t)(a.D / Ops::kLanes);
+  const int64_t first = (int64_t)blockIdx.x * kEncodeThreads;  // first item of this block
+  const int64_t g0 = first / Dv;
+  const uint32_t t = (uint32_t)(first - g0 * Dv) + threadIdx.x;
+  const uint32_t dg = t / Dv;
+  const uint32_t v = t - dg * Dv;
+  const int64_t g = g0 + dg;
+  if (g >= a.G) return;
+
+  const V* in = reinterpret_cast<const V*>(a.X + g * a.x_gs) + v;
+  V* out = reinterpret_cast<V*>(a.Xt + g * a.o_gs) + v;
+  const int64_t in_rs = a.x_rs / Ops::kLanes;
+  const int64_t out_rs = a.o_rs / Ops::kLanes;
+
+  V x[K];
+#pragma unroll
+  for (int j = 0; j < K; ++j) x[j] = ld_stream(in + j * in_rs);
+
+  const int W = a.W;
+  for (int i = 0; i < W; ++i) {
+    const float* wi = tab.w + i * K;
+    V acc = Ops::mul(wi[0], x[0]);
+#pragma unroll
+    for (int j = 1; j < K; ++j) acc = Ops::fma(wi[j], x[j], acc);
+    st_stream(out + i * out_rs, acc);
+  }
+}
+
+template <int K, typename V>
+cudaError_t launch_one(const EncodeArgs& a, const EncodeTables& tab, cudaStream_t stream) {
+  const int64_t Dv = a.D / VecOps<V>::kLanes;
+  const int64_t items = a.G * Dv;
+  const int64_t blocks = (items + kEncodeThreads - 1) / kEncodeThreads;
+  if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+  encode_kernel<K, V><<<(unsigned)blocks, kEncodeThreads, 0, stream>>>(a, tab);
+  count_launch();
+  return cudaGetLastError();
+}
+
+template <typename V, int K = 1>
+cudaError_t dispatch_k(const EncodeArgs& a, const EncodeTables& tab, cudaStream_t stream) {
+  if constexpr (K > kMaxK) {
+    return cudaErrorInvalidValue;
+  } else {
+    if (a.K == K) return launch_one<K, V>(a, tab, stream);
+    return dispatch_k<V, K + 1>(a, tab, stream);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_encode(const EncodeArgs& a, cudaStream_t stream) {
+  if (a.G == 0) return cudaSuccess;
+  EncodeTables tab;
+  build_encode_tables(a.K, a.W, &tab);
+  const bool vec = aligned16(a.X) && aligned16(a.Xt) && a.D % 4 == 0 && a.x_gs % 4 == 0 && a.x_rs % 4 == 0 &&
+                   a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  if (vec) return dispatch_k<float4>(a, tab, stream);
+  return dispatch_k<float>(a, tab, stream);
+}
+
+}  // namespace approxifer

@@ -1,0 +1,76 @@
+// Host-side node tables (see tables.h).
+#include "tables.h"
+
+#include <cmath>
+#include <cstring>
+
+namespace approxifer {
+
+namespace {
+
+const long double kPi = 3.14159265358979323846264338327950288L;
+
+// sin(pi * p / den) for integers |p| <= den, den > 0.  The argument is folded
+// into [0, 1/4] in integer arithmetic first, so the only rounding is that of
+// one division and one sin/cos of a small argument.
+long double sinpi_ratio(long long p, long long den) {
+  if (p < 0) return -sinpi_ratio(-p, den);
+  if (2 * p > den) p = den - p;  // sin(pi x) = sin(pi (1 - x))
+  if (4 * p > den)               // sin(pi x) = cos(pi (1/2 - x))
+    return cosl(kPi * (long double)(den - 2 * p) / (long double)(2 * den));
+  return sinl(kPi * (long double)p / (long double)den);
+}
+
+}  // namespace
+
+long double node_gap(int K, int W, int j, int i) {
+  // a = pi (2j+1)/(2K), b = pi i/(W-1):
+  //   (a+b)/2 = pi [(2j+1)(W-1) + 2Ki] / (4K(W-1)),  (a-b)/2 likewise with a minus.
+  const long long den = 4LL * K * (W - 1);
+  const long long s = (long long)(2 * j + 1) * (W - 1);
+  const long long t = 2LL * K * i;
+  return -2.0L * sinpi_ratio(s + t, den) * sinpi_ratio(s - t, den);
+}
+
+void build_encode_tables(int K, int W, EncodeTables* t) {
+  std::memset(t, 0, sizeof(*t));
+  for (int i = 0; i < W; ++i) {
+    int hit = -1;
+    for (int j = 0; j < K; ++j)
+      if (nodes_coincide(K, W, j, i)) hit = j;
+    if (hit >= 0) {  // u passes through the query: the row is one-hot
+      t->w[i * K + hit] = 1.0f;
+      continue;
+    }
+    // l_j(beta_i) = [(-1)^j/(beta_i - alpha_j)] / sum_k (-1)^k/(beta_i - alpha_k)
+    long double term[kMaxK], den = 0.0L;
+    for (int j = 0; j < K; ++j) {
+      term[j] = ((j & 1) ? -1.0L : 1.0L) / (-node_gap(K, W, j, i));
+      den += term[j];
+    }
+    for (int j = 0; j < K; ++j) t->w[i * K + j] = (float)(term[j] / den);
+  }
+}
+
+void build_decode_tables(int K, int W, DecodeTables* t) {
+  std::memset(t, 0, sizeof(*t));
+  for (int j = 0; j < K; ++j) t->coin[j] = -1;
+  for (int i = 0; i < W; ++i)
+    for (int j = 0; j < K; ++j) {
+      if (nodes_coincide(K, W, j, i)) {
+        t->coin[j] = (int8_t)i;
+        t->any_coin = 1;
+        t->rg[i * K + j] = 0.0f;
+      } else {
+        t->rg[i * K + j] = (float)(1.0L / node_gap(K, W, j, i));
+      }
+    }
+}
+
+void build_locate_tables(int W, LocateTables* t) {
+  std::memset(t, 0, sizeof(*t));
+  // beta_i = cos(pi i/(W-1)) = sin(pi (1/2 - i/(W-1)))
+  for (int i = 0; i < W; ++i) t->beta[i] = (double)sinpi_ratio((long long)(W - 1) - 2 * i, 2LL * (W - 1));
+}
+
+}  // namespace approxifer

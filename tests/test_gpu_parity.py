@@ -1,0 +1,356 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU
+oracle on the same seeded inputs, element by element.
+
+Tolerances (fp32 kernels vs fp64 oracle):
+  encode : max |Xt_gpu - Xt_oracle| <= 1e-5 * max |X|  over the tensor
+  decode : per group, max |Yh_gpu - Yh_oracle| <= 1e-4 * max |Yh_oracle| of that group
+  mask compaction (n_used, worker lists) and the located set: bit-exact
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2109_09868_b200 as ap
+from paper_2109_09868_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+ENC_TOL = 1e-5
+DEC_TOL = 1e-4
+CANARY = 1234.5
+
+
+def dev():
+    return torch.device("cuda:0")
+
+
+def check_encode(K, W, X_cpu, Xt_gpu):
+    ref = oracle.encode(K, W, X_cpu.numpy())
+    err = np.abs(Xt_gpu.cpu().numpy().astype(np.float64) - ref).max() if ref.size else 0.0
+    scale = float(X_cpu.abs().max()) if X_cpu.numel() else 1.0
+    assert err <= ENC_TOL * scale, (K, W, err, scale)
+    return err
+
+
+def check_decode(K, W, Yt_cpu, mask_np, Yh_gpu, n_used=None, status=None, flags=0):
+    ref, n_ref, st_ref = oracle.decode(K, W, Yt_cpu.numpy(), mask_np, flags)
+    got = Yh_gpu.cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    err = np.abs(got - ref).reshape(len(mask_np), -1).max(axis=1)
+    scale = np.abs(ref).reshape(len(mask_np), -1).max(axis=1)
+    bad = err > DEC_TOL * np.maximum(scale, 1e-30)
+    bad &= ~((scale == 0) & (err == 0))
+    assert not bad.any(), (K, W, int(bad.sum()), float(err[bad].max()), float(scale[bad].min()))
+    if n_used is not None:
+        np.testing.assert_array_equal(n_used.cpu().numpy(), n_ref)
+    if status is not None:
+        np.testing.assert_array_equal(status.cpu().numpy().view(np.uint32), st_ref)
+    return float((err / np.maximum(scale, 1e-30)).max())
+
+
+# ------------------------------------------------------------------- encode
+
+ENCODE_SHAPES = [
+    (4, 5, 256, 784),    # workload 1
+    (8, 12, 7, 3072),    # workload 2 shape
+    (12, 20, 2, 150528),  # workload 3 shape, several tiles
+    (16, 24, 33, 32),
+    (8, 24, 65, 64),
+    (3, 7, 5, 1000),     # coincident nodes: rows 1, 3, 5 copy queries 0, 1, 2
+    (1, 2, 3, 8),
+    (1, 9, 3, 12),
+    (2, 5, 4, 16),
+    (32, 32, 3, 260),
+    (31, 2, 2, 4),
+    (5, 32, 2, 516),
+    (7, 9, 300, 4),      # D = 4: one column per group, many groups per block
+]
+
+
+@pytest.mark.parametrize("K,W,G,D", ENCODE_SHAPES)
+def test_encode_matches_oracle(K, W, G, D):
+    g = torch.Generator().manual_seed(K * 1000 + W)
+    X = torch.rand((G, K, D), generator=g) * 2 - 0.5
+    p = ap.make_params(K, W)
+    Xt = ap.approxifer_encode(p, X.to(dev()))
+    torch.cuda.synchronize()
+    check_encode(K, W, X, Xt)
+    if (K, W) == (3, 7):
+        for (j, i) in [(0, 1), (1, 3), (2, 5)]:
+            assert torch.equal(Xt[:, i].cpu(), X[:, j])
+    if K == 1:
+        for i in range(W):
+            assert torch.equal(Xt[:, i].cpu(), X[:, 0])
+
+
+@pytest.mark.parametrize("K,W,G,D", [(4, 5, 9, 783), (8, 12, 3, 3071), (3, 7, 4, 1), (12, 20, 2, 1001), (5, 6, 40, 3)])
+def test_encode_odd_lengths_take_the_elementwise_path(K, W, G, D):
+    g = torch.Generator().manual_seed(D)
+    X = torch.rand((G, K, D), generator=g)
+    Xt = ap.approxifer_encode(ap.make_params(K, W), X.to(dev()))
+    check_encode(K, W, X, Xt)
+
+
+def test_encode_misaligned_strided_and_guarded_buffers():
+    K, W, G, D = 8, 12, 6, 260
+    g = torch.Generator().manual_seed(5)
+    X = torch.rand((G, K, D), generator=g)
+    p = ap.make_params(K, W)
+    # (a) base pointers off by one float: not 16-byte aligned
+    xin = torch.zeros(G * K * D + 1, device=dev())
+    xin[1:] = X.flatten().to(dev())
+    out = torch.full((G * W * D + 9,), CANARY, device=dev())
+    Xt = ap.approxifer_encode(p, xin[1:].view(G, K, D), out[5 : 5 + G * W * D].view(G, W, D))
+    check_encode(K, W, X, Xt)
+    assert bool((out[:5] == CANARY).all()) and bool((out[5 + G * W * D :] == CANARY).all())
+    # (b) padded rows (row stride > D) on both sides, canaries in the padding
+    pad = 12
+    xin2 = torch.full((G, K, D + pad), CANARY, device=dev())
+    xin2[:, :, :D] = X.to(dev())
+    out2 = torch.full((G, W, D + pad), CANARY, device=dev())
+    ap.approxifer_encode(p, xin2[:, :, :D], out2[:, :, :D])
+    check_encode(K, W, X, out2[:, :, :D])
+    assert bool((out2[:, :, D:] == CANARY).all())
+    # (c) worker-major output [W][G][D]
+    out3 = torch.empty((W, G, D), device=dev())
+    ap.approxifer_encode(p, X.to(dev()), out3.permute(1, 0, 2))
+    check_encode(K, W, X, out3.permute(1, 0, 2))
+    # (d) G = 0
+    ap.approxifer_encode(p, torch.empty((0, K, D), device=dev()))
+
+
+def test_encode_weights_on_device_match_oracle():
+    for (K, W) in [(4, 5), (8, 12), (12, 20), (16, 24), (8, 24), (3, 7), (32, 32), (1, 2), (2, 5), (4, 9)]:
+        w = ap.approxifer_debug_weights(ap.make_params(K, W), which=0).cpu().numpy().astype(np.float64)
+        ref = oracle.encode_weights(K, W)
+        assert np.abs(w - ref).max() <= 1.2e-7 * max(1.0, np.abs(ref).max()), (K, W)
+        for i in range(W):
+            for j in range(K):
+                if oracle.coincident(K, W, j, i):
+                    assert w[i, j] == 1.0 and np.abs(w[i]).sum() == 1.0
+
+
+# ------------------------------------------------------------------- decode
+
+def random_masks(W, G, rng, min_present=0):
+    m = rng.integers(0, 2**W, size=G, dtype=np.uint64)
+    for g in range(G):
+        while bin(int(m[g])).count("1") < min_present:
+            m[g] |= np.uint64(1) << np.uint64(rng.integers(0, W))
+    return m.astype(np.uint32)
+
+
+DECODE_SHAPES = [
+    (4, 5, 256, 10),
+    (8, 12, 300, 10),
+    (12, 20, 9, 1000),
+    (16, 24, 21, 1000),
+    (8, 24, 130, 10),
+    (3, 7, 64, 36),     # coincident nodes
+    (1, 2, 8, 4),
+    (2, 5, 32, 8),      # alpha = +-sqrt(2)/2 coincide with beta_1, beta_3
+    (4, 9, 40, 12),
+    (32, 32, 5, 260),
+    (5, 32, 6, 513),
+    (9, 11, 50, 1),
+]
+
+
+@pytest.mark.parametrize("K,W,G,C", DECODE_SHAPES)
+@pytest.mark.parametrize("flags", [0, 1])
+def test_decode_matches_oracle(K, W, G, C, flags):
+    rng = np.random.default_rng(K * 100 + W + flags)
+    g = torch.Generator().manual_seed(K * 100 + W)
+    Yt = torch.randn((G, W, C), generator=g)
+    mask = random_masks(W, G, rng, min_present=(0 if flags == 0 else max(W - 2, 1)))
+    mask[0] = 2**W - 1
+    if flags == 1:
+        # the literal sign (-1)^i has real poles when the used workers are not a
+        # contiguous run; keep only masks whose weights stay moderate
+        for gi in range(G):
+            w_lit, _ = oracle.decode_weights(K, W, int(mask[gi]), 1)
+            if np.abs(w_lit).sum(axis=1).max() > 30.0:
+                mask[gi] = 2**W - 1
+    if flags == 0 and G > 3:
+        mask[1] = 0
+        mask[2] = 1 << (W - 1)
+        mask[3] |= np.uint32((0xFFFFFFFF << W) & 0xFFFFFFFF)  # bits beyond W must be ignored
+    p = ap.make_params(K, W, 0, flags)
+    n_used = torch.empty(G, dtype=torch.int32, device=dev())
+    status = torch.empty(G, dtype=torch.int32, device=dev())
+    Yh = ap.approxifer_decode(p, Yt.to(dev()), ap.mask_tensor(mask), n_used=n_used, status=status)
+    check_decode(K, W, Yt, mask, Yh, n_used, status, flags)
+
+
+@pytest.mark.parametrize("K,W", [(2, 3), (3, 6), (4, 8), (3, 7), (2, 5)])
+def test_decode_all_masks_exhaustively(K, W):
+    G, C = 2**W, 12
+    g = torch.Generator().manual_seed(W)
+    Yt = torch.randn((G, W, C), generator=g)
+    mask = np.arange(G, dtype=np.uint32)
+    n_used = torch.empty(G, dtype=torch.int32, device=dev())
+    status = torch.empty(G, dtype=torch.int32, device=dev())
+    Yh = ap.approxifer_decode(ap.make_params(K, W), Yt.to(dev()), ap.mask_tensor(mask), n_used=n_used, status=status)
+    check_decode(K, W, Yt, mask, Yh, n_used, status)
+    # compaction through the weight hook: worker lists are bit-exact
+    for m in (1, 5, G - 1, G // 2 + 3):
+        w, idx = ap.approxifer_debug_weights(ap.make_params(K, W), mask=m, which=1)
+        w_ref, F = oracle.decode_weights(K, W, m)
+        assert idx.cpu().tolist() == F
+        assert np.abs(w.cpu().numpy() - w_ref).max() <= 2e-6 * max(1.0, np.abs(w_ref).max())
+
+
+def test_decode_ignores_garbage_in_absent_rows_and_copies_at_coincident_nodes():
+    K, W, G, C = 3, 7, 16, 20
+    rng = np.random.default_rng(3)
+    g = torch.Generator().manual_seed(3)
+    Yt = torch.randn((G, W, C), generator=g)
+    mask = random_masks(W, G, rng, min_present=2)
+    mask[0] = 0x7F
+    dirty = Yt.clone()
+    for gi in range(G):
+        for i in range(W):
+            if not (int(mask[gi]) >> i) & 1:
+                dirty[gi, i] = float("nan")
+    p = ap.make_params(K, W)
+    a = ap.approxifer_decode(p, Yt.to(dev()), ap.mask_tensor(mask))
+    b = ap.approxifer_decode(p, dirty.to(dev()), ap.mask_tensor(mask))
+    assert torch.equal(a, b)
+    check_decode(K, W, Yt, mask, a)
+    for (j, i) in [(0, 1), (1, 3), (2, 5)]:
+        for gi in range(G):
+            if (int(mask[gi]) >> i) & 1:
+                assert torch.equal(a[gi, j].cpu(), Yt[gi, i])
+
+
+def test_decode_misaligned_strided_and_guarded_buffers():
+    K, W, G, C = 8, 12, 10, 100
+    rng = np.random.default_rng(8)
+    g = torch.Generator().manual_seed(8)
+    Yt = torch.randn((G, W, C), generator=g)
+    mask = random_masks(W, G, rng, min_present=1)
+    p = ap.make_params(K, W)
+    yin = torch.zeros(G * W * C + 3, device=dev())
+    yin[3:] = Yt.flatten().to(dev())
+    out = torch.full((G * K * C + 8,), CANARY, device=dev())
+    Yh = ap.approxifer_decode(p, yin[3:].view(G, W, C), ap.mask_tensor(mask), out[2 : 2 + G * K * C].view(G, K, C))
+    check_decode(K, W, Yt, mask, Yh)
+    assert bool((out[:2] == CANARY).all()) and bool((out[2 + G * K * C :] == CANARY).all())
+    pad = 4
+    yin2 = torch.full((G, W, C + pad), float("nan"), device=dev())
+    yin2[:, :, :C] = Yt.to(dev())
+    out2 = torch.full((G, K, C + pad), CANARY, device=dev())
+    ap.approxifer_decode(p, yin2[:, :, :C], ap.mask_tensor(mask), out2[:, :, :C])
+    check_decode(K, W, Yt, mask, out2[:, :, :C])
+    assert bool((out2[:, :, C:] == CANARY).all())
+
+
+# ------------------------------------------------------------------- locate
+
+def linear_case(K, W, E, S, G, C, seed, softmax=False, sigma=10.0, d_in=16):
+    """Honest predictions = linear (optionally + softmax) model of the ORACLE's
+    coded queries, E corrupted workers among the W-S present."""
+    rng = np.random.default_rng(seed)
+    X = rng.random((G, K, d_in), dtype=np.float32)
+    M = rng.standard_normal((d_in, C)) / np.sqrt(d_in)
+    Y = oracle.encode(K, W, X) @ M
+    if softmax:
+        Y = np.exp(Y - Y.max(axis=-1, keepdims=True))
+        Y /= Y.sum(axis=-1, keepdims=True)
+    Y = Y.astype(np.float32)
+    mask = np.empty(G, dtype=np.uint32)
+    truth = np.empty((G, E), dtype=np.int32)
+    for g in range(G):
+        present = np.sort(rng.choice(W, size=W - S, replace=False))
+        mask[g] = sum(1 << int(i) for i in present)
+        bad = np.sort(rng.choice(present, size=E, replace=False))
+        truth[g] = bad
+        Y[g, bad] += (sigma * rng.standard_normal((E, C))).astype(np.float32)
+    return torch.from_numpy(Y), mask, truth
+
+
+def run_locate(K, W, E, Yt, mask):
+    G = Yt.shape[0]
+    status = torch.empty(G, dtype=torch.int32, device=dev())
+    adv, trusted = ap.approxifer_locate(ap.make_params(K, W, E), Yt.to(dev()), ap.mask_tensor(mask), status=status)
+    torch.cuda.synchronize()
+    return adv.cpu().numpy(), trusted.cpu().numpy().view(np.uint32), status.cpu().numpy().view(np.uint32)
+
+
+def compare_locate(K, W, E, Yt, mask, allow_fragile=False):
+    ref = oracle.locate(K, W, E, Yt.numpy(), mask)
+    adv, trusted, status = run_locate(K, W, E, Yt, mask)
+    solid = (ref["min_gap"] > 1.0 + 1e-6) & (ref["vote_margin"] > 0) & ((ref["status"] & oracle.ST_ORACLE_RANK_DEFICIENT) == 0)
+    solid |= (ref["status"] & oracle.ST_LOCATE_UNDERDETERMINED) != 0
+    if not allow_fragile:
+        assert solid.all(), "workload has near-tied groups: %d" % int((~solid).sum())
+    np.testing.assert_array_equal(adv[solid], ref["adv"][solid])
+    np.testing.assert_array_equal(trusted[solid], ref["trusted"][solid])
+    np.testing.assert_array_equal(status[solid], ref["status"][solid] & 0xFF)
+    # whatever was returned is always a valid answer: E distinct present workers, ascending
+    for g in range(len(mask)):
+        if ref["status"][g] & oracle.ST_LOCATE_UNDERDETERMINED:
+            continue
+        row = adv[g]
+        assert np.all(np.diff(row) > 0) and all((int(mask[g]) >> int(i)) & 1 for i in row)
+        assert int(trusted[g]) == (int(mask[g]) & (2**W - 1)) & ~sum(1 << int(i) for i in row)
+    return ref, adv, int((~solid).sum())
+
+
+@pytest.mark.parametrize("K,E,S,W", [(8, 2, 2, 24), (2, 1, 0, 6), (3, 2, 1, 12), (4, 1, 2, 12), (12, 2, 0, 28),
+                                     (6, 3, 1, 20), (1, 1, 0, 4), (13, 3, 0, 32), (8, 2, 0, 20), (2, 1, 3, 9)])
+def test_locate_matches_oracle_and_finds_injected_errors(K, E, S, W):
+    G, C = 96, 10
+    Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=K * 31 + E)
+    ref, adv, _ = compare_locate(K, W, E, Yt, mask)
+    if W % 2 == 0:  # no node at 0: Theorem 1 guarantees exact location for a rational model
+        np.testing.assert_array_equal(adv, truth)
+
+
+def test_locate_softmax_model_and_noise_scales():
+    K, E, S, W = 8, 2, 2, 24
+    for sigma in (1.0, 10.0, 100.0):
+        Yt, mask, truth = linear_case(K, W, E, S, 256, 10, seed=int(sigma), softmax=True, sigma=sigma)
+        ref, adv, fragile = compare_locate(K, W, E, Yt, mask, allow_fragile=True)
+        assert fragile <= 8
+        assert (adv == truth).all(axis=1).mean() > 0.9
+
+
+def test_locate_many_classes_one_class_and_underdetermined_groups():
+    K, E, S, W = 4, 1, 1, 12
+    Yt, mask, truth = linear_case(K, W, E, S, 24, 1000, seed=77)
+    compare_locate(K, W, E, Yt, mask)
+    Yt1, mask1, _ = linear_case(K, W, E, S, 40, 1, seed=78)
+    mask1[::4] = 0b000111111111  # 9 < 2(K+E) = 10 workers -> nothing located
+    mask1[1] = 0
+    ref, adv, _ = compare_locate(K, W, E, Yt1, mask1)
+    assert (adv[::4] == -1).all() and adv[1, 0] == -1
+    # a class whose predictions are exactly zero leaves Q = 1: the lowest workers are picked
+    Z = torch.zeros((3, W, 2))
+    full = np.full(3, 2**W - 1, dtype=np.uint32)
+    ref, adv, _ = compare_locate(K, W, E, Z, full, allow_fragile=True)
+    assert (adv == 0).all() and (ref["adv"] == 0).all()
+
+
+def test_locate_then_decode_pipeline_matches_oracle():
+    K, E, S, W, G, C = 8, 2, 2, 24, 200, 10
+    Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=5)
+    p = ap.make_params(K, W, E)
+    adv, trusted = ap.approxifer_locate(p, Yt.to(dev()), ap.mask_tensor(mask))
+    n_used = torch.empty(G, dtype=torch.int32, device=dev())
+    Yh = ap.approxifer_decode(p, Yt.to(dev()), trusted, n_used=n_used)
+    ref = oracle.locate(K, W, E, Yt.numpy(), mask)
+    np.testing.assert_array_equal(trusted.cpu().numpy().view(np.uint32), ref["trusted"])
+    check_decode(K, W, Yt, ref["trusted"], Yh, n_used)
+    assert bool((n_used == W - S - E).all())
+
+
+def test_strided_predictions_for_locate():
+    K, E, S, W, G, C = 3, 1, 0, 8, 20, 7
+    Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=9)
+    big = torch.full((G, W, C + 5), float("nan"))
+    big[:, :, :C] = Yt
+    adv, trusted = ap.approxifer_locate(ap.make_params(K, W, E), big.to(dev())[:, :, :C], ap.mask_tensor(mask))
+    ref = oracle.locate(K, W, E, Yt.numpy(), mask)
+    np.testing.assert_array_equal(adv.cpu().numpy(), ref["adv"])
