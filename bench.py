@@ -85,7 +85,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -122,7 +122,7 @@ class ClockSampler:
 
 # ------------------------------------------------------------------- CPU oracle
 
-def time_oracle(sample_groups: int = 2048, min_seconds: float = 10.0, max_reps: int = 40):
+def time_oracle(sample_groups: int = 4096, min_seconds: float = 12.0, max_reps: int = 2000):
     """Times the fp64 CPU checker, as it stands, on a bounded sample of the
     headline workload (encode + decode of `sample_groups` groups, repeated)."""
     import oracle
@@ -361,7 +361,7 @@ def run_e2e(ap, dev, w, mask_np, steps, warmup):
 def main():
     ap_ = argparse.ArgumentParser()
     ap_.add_argument("--gpus", type=int, default=1)
-    ap_.add_argument("--steps", type=int, default=20)
+    ap_.add_argument("--steps", type=int, default=400)
     ap_.add_argument("--warmup", type=int, default=3)
     ap_.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap_.add_argument("--no-others", action="store_true", help="skip the per-configuration kernel figures")
@@ -424,6 +424,7 @@ def main():
         dist.barrier()
     torch.cuda.synchronize()
     sampler.start()
+    time.sleep(0.2)  # let the sampler take its first readings
     launches0 = ap.launch_count()
     e_begin.record()
     for s in range(args.steps):
