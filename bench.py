@@ -301,6 +301,46 @@ def other_workloads(ap, dev, peak):
     return out
 
 
+def run_case(ap, dev, args):
+    """One kernel of one configuration, timed alone (CUDA events per launch)."""
+    cfg = int(args.case[-1])
+    op = args.case[:-1]
+    w = wl.workload(cfg, args.groups)
+    p = ap.make_params(w.K, w.W, w.E)
+    iters = max(args.steps, 1)
+    warm = max(args.warmup, 1)
+    if op == "encode":
+        X = wl.queries(w, dev)
+        Xt = torch.empty((w.G, w.W, w.D), device=dev)
+        med, mn = time_launches(lambda: ap.approxifer_encode(p, X, Xt), warm, iters)
+        nbytes = encode_bytes(w)
+    else:
+        if cfg in (2, 3):
+            Yt = wl.gaussian_predictions(w, dev)
+        else:
+            Xc = ap.approxifer_encode(p, wl.queries(w, dev))
+            Yt = torch.empty((w.G, w.W, w.C), device=dev)
+            for s in range(0, w.G, 16384):
+                Yt[s:s + 16384] = wl.apply_model(w, Xc[s:s + 16384])
+            del Xc
+        m = wl.masks(w)
+        if cfg == 5:
+            wl.corrupt(w, Yt, wl.adversaries(w, m))
+        mt = ap.mask_tensor(m, dev)
+        if op == "locate":
+            adv = torch.empty((w.G, w.E), dtype=torch.int32, device=dev)
+            trusted = torch.empty((w.G,), dtype=torch.int32, device=dev)
+            med, mn = time_launches(lambda: ap.approxifer_locate(p, Yt, mt, adv, trusted), warm, iters)
+            nbytes = locate_bytes(w, m)
+        else:
+            Yh = torch.empty((w.G, w.K, w.C), device=dev)
+            med, mn = time_launches(lambda: ap.approxifer_decode(p, Yt, mt, Yh), warm, iters)
+            nbytes = decode_bytes(w, m)
+    return {"case": args.case, "groups": w.G, "dec_config": args.dec_config, "ms": med, "ms_min": mn,
+            "GB_per_s": nbytes / med / 1e6, "groups_per_s": w.G / med * 1e3, "algorithmic_GB": nbytes / 1e9,
+            "wait_timeouts": ap.device_wait_timeouts()}
+
+
 def run_e2e(ap, dev, w, mask_np, steps, warmup):
     """Same metric through the public API with HOST buffers: every step copies
     the queries and the coded predictions from pinned host memory, runs encode
@@ -368,6 +408,9 @@ def main():
     ap_.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap_.add_argument("--no-cpu", action="store_true", help="skip timing the CPU checker")
     ap_.add_argument("--groups", type=int, default=None, help="override the number of groups (profiling only)")
+    ap_.add_argument("--case", default=None, choices=["decode3", "decode4", "locate5", "decode5", "decode2", "encode3"],
+                     help="time one kernel of another configuration alone (tuning / profiling) and print a short JSON line")
+    ap_.add_argument("--dec-config", default=None, help="stages,ctas_per_sm,disable,cols,split for the wide decoder (tuning)")
     args = ap_.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -388,6 +431,12 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     import paper_2109_09868_b200 as ap
+
+    if args.dec_config:
+        ap.debug_decode_config(*[int(v) for v in args.dec_config.split(",")])
+    if args.case:
+        print(json.dumps(run_case(ap, dev, args)), flush=True)
+        return
 
     # CPU baseline first (rank 0, N = 1 only), before the GPU gets busy
     cpu = None

@@ -76,7 +76,7 @@ typedef struct approxifer_params {
  *     l_j(z) = [(-1)^j/(z-alpha_j)] / sum_k (-1)^k/(z-alpha_k).
  * If beta_i equals some alpha_j (exactly when (2j+1)(W-1) == 2Ki) the row is
  * the limit value X[g][j][:].
- *   X   in,  [G][K][D], strides x_gstride >= ?, x_rstride >= D (elements)
+ *   X   in,  [G][K][D], x_rstride >= D, x_gstride >= 0 (elements)
  *   Xt  out, [G][W][D], strides xt_gstride, xt_rstride >= D; a worker-major
  *            layout [W][G][D] is expressed as xt_gstride = D, xt_rstride = G*D.
  * fp32 accumulation, one fused multiply-add per term, j ascending.
@@ -139,6 +139,26 @@ int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C,
  */
 int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int which,
                              float* w, int32_t* idx, int32_t* n, void* cuda_stream);
+
+/*
+ * Test / tuning hook for the wide-payload decoder (C >= 512, 128-bit path,
+ * default sign), which stages the rows of present workers through shared memory
+ * with bulk asynchronous copies.  stages: 0 (as many as fit, at most 4) or an
+ * upper bound >= 2 on the ring depth; ctas_per_sm: 0 (automatic) or an upper
+ * bound; disable != 0 routes every decode through the register-staged kernel;
+ * cols: 0 (automatic), 64 or 128 16-byte columns per work item; split: 0
+ * (automatic), 2 or 4 thread groups sharing the K queries of a column.
+ * Process-wide, not thread-safe; results are bit-identical for every setting.
+ */
+int approxifer_debug_decode_config(int stages, int ctas_per_sm, int disable, int cols, int split);
+
+/*
+ * Every wait on an asynchronous copy inside the kernels is bounded.  Returns how
+ * many such waits have given up on the current device since the library was
+ * loaded (0 in a correct run; the affected groups' outputs are then
+ * unspecified), or -1 if the counter cannot be read.  Synchronises the device.
+ */
+int64_t approxifer_device_wait_timeouts(void);
 
 /* Human-readable text for a return code (static storage). */
 const char* approxifer_strerror(int code);

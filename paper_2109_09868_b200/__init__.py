@@ -12,6 +12,8 @@ from .binding import (  # noqa: F401
     approxifer_encode,
     approxifer_locate,
     approxifer_params,
+    debug_decode_config,
+    device_wait_timeouts,
     launch_count,
     library_path,
     load,

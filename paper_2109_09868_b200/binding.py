@@ -30,6 +30,8 @@ EXPORTS = (
     "approxifer_strerror",
     "approxifer_version",
     "approxifer_launch_count",
+    "approxifer_debug_decode_config",
+    "approxifer_device_wait_timeouts",
 )
 
 
@@ -80,6 +82,9 @@ def load() -> ctypes.CDLL:
     lib.approxifer_strerror.restype = c_char_p
     lib.approxifer_version.restype = c_int
     lib.approxifer_launch_count.restype = c_int64
+    lib.approxifer_debug_decode_config.argtypes = [c_int, c_int, c_int, c_int, c_int]
+    lib.approxifer_debug_decode_config.restype = c_int
+    lib.approxifer_device_wait_timeouts.restype = c_int64
     del pf, pu, pi
     _lib = lib
     return lib
@@ -95,6 +100,16 @@ def version() -> int:
 
 def launch_count() -> int:
     return int(load().approxifer_launch_count())
+
+
+def debug_decode_config(stages: int = 0, ctas_per_sm: int = 0, disable: int = 0, cols: int = 0, split: int = 0) -> None:
+    rc = load().approxifer_debug_decode_config(int(stages), int(ctas_per_sm), int(disable), int(cols), int(split))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_debug_decode_config")
+
+
+def device_wait_timeouts() -> int:
+    return int(load().approxifer_device_wait_timeouts())
 
 
 def make_params(K: int, W: int, E: int = 0, flags: int = 0) -> approxifer_params:

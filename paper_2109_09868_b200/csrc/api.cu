@@ -91,6 +91,20 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
                                         static_cast<cudaStream_t>(cuda_stream)));
 }
 
+int approxifer_debug_decode_config(int stages, int ctas_per_sm, int disable, int cols, int split) {
+  if (stages < 0 || stages == 1 || ctas_per_sm < 0 || (cols != 0 && cols != 64 && cols != 128) ||
+      (split != 0 && split != 2 && split != 4))
+    return APPROXIFER_E_PARAM;
+  decode_staged_config(stages, ctas_per_sm, disable, cols, split);
+  return APPROXIFER_OK;
+}
+
+int64_t approxifer_device_wait_timeouts(void) {
+  unsigned int n = 0;
+  if (read_decode_wait_timeouts(&n) != cudaSuccess) return -1;
+  return (int64_t)n;
+}
+
 const char* approxifer_strerror(int code) {
   switch (code) {
     case APPROXIFER_OK: return "ok";

@@ -54,6 +54,12 @@ cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream);
 cudaError_t launch_debug_weights(int K, int W, uint32_t flags, uint32_t mask, int which, float* w, int32_t* idx,
                                  int32_t* n, cudaStream_t stream);
 
+// Wide-payload decoder (bulk-copy staged); see decode_staged.cu.
+bool decode_staged_eligible(const DecodeArgs& a);
+cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream);
+void decode_staged_config(int stages, int ctas_per_sm, int disable, int cols, int split);
+cudaError_t read_decode_wait_timeouts(unsigned int* out);
+
 void count_launch(int n = 1);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -1,0 +1,436 @@
+// ApproxIFER decoder, wide-payload variant (Section 3, "Decoding", step 2).
+//
+// Same arithmetic as decode_kernel (barycentric numerator / denominator over
+// the workers present in the mask, terms added in ascending worker order),
+// different data movement: persistent CTAs pull the rows of PRESENT workers
+// only into a shared-memory ring with bulk asynchronous copies
+// (cp.async.bulk global -> shared, completion counted on an mbarrier), so the
+// HBM reads of the next work items are in flight while the current item is
+// reduced from shared memory.  Nothing waits on a register-staged load and the
+// register file holds only the accumulators.
+//
+// A work item is (group, tile of COLS 16-byte columns).  2*COLS compute threads
+// work on it: thread = (half, column); half h forms the queries
+// j = h*KT .. h*KT+KT-1 (KT = ceil(K/SPLIT)), so two warps share each column's
+// payload but every thread keeps only KT accumulators per payload element,
+// which doubles the warps per byte of ring.  The FMAs are packed
+// (fma.rn.f32x2: the weights of two adjacent queries times one payload
+// element, each half an ordinary round-to-nearest fp32 FMA).  One more warp is
+// the producer: for each item it waits for a free ring slot, writes the item's
+// signed weights (by rank) and K reciprocal denominators into the slot, and
+// starts the copies of the present rows; slots are handed over and back
+// through "full" / "empty" mbarriers, so producer and compute warps never meet
+// at a CTA-wide barrier.  Every wait is bounded.  Items are dealt round-robin
+// to the CTAs.  No cluster multicast is used.
+#include "common.cuh"
+
+namespace approxifer {
+
+__device__ unsigned int g_decode_wait_timeouts = 0;  // bounded waits that gave up (never, in a correct run)
+
+namespace {
+
+constexpr int kMaxStages = 4;
+constexpr uint32_t kWaitLimit = 1u << 22;  // try_wait attempts before a wait gives up
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within kWaitLimit attempts.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kWaitLimit; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// 1-D bulk copy global -> this CTA's shared memory; src, dst and bytes are multiples of 16.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;  // two independent round-to-nearest fp32 FMAs on the packed halves
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t dup(uint32_t v) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %1};" : "=l"(d) : "r"(v));
+  return d;
+}
+__device__ __forceinline__ float lo_f(uint64_t v) { return __uint_as_float((uint32_t)v); }
+__device__ __forceinline__ float hi_f(uint64_t v) { return __uint_as_float((uint32_t)(v >> 32)); }
+
+struct StagedPlan {
+  int32_t tiles;       // column tiles per group
+  int32_t stages;      // ring depth
+  int64_t n_items;     // G * tiles
+};
+
+constexpr int kWeightsOff = 16 + 128;  // header, reciprocal denominators
+__host__ __device__ constexpr int ktp4(int KT) { return (KT + 3) / 4 * 4;  }  // weights of one half, padded to float4s
+// Per-slot item block: n (16 B) | 1/denominators (32 floats) | weights of the present workers, by rank:
+//   float w[r][h][jj] = s_r / (alpha_j - beta_{F[r]}), j = h*KT + jj (0 beyond K or KT).
+__host__ __device__ constexpr int meta_bytes(int W, int KT, int SPLIT) { return (kWeightsOff + W * SPLIT * ktp4(KT) * 4 + 127) / 128 * 128; }
+constexpr int kTableOff = 128;  // float rg[W][K] after the mbarriers and the abort flag
+__host__ __device__ constexpr int slots_off(int W, int K) { return (kTableOff + W * (K | 1) * 4 + 127) / 128 * 128; }
+__host__ __device__ constexpr int slot_bytes(int W, int KT, int SPLIT, int COLS) { return meta_bytes(W, KT, SPLIT) + W * COLS * 16; }
+__host__ __device__ constexpr int min_ctas(int KT, int threads) { return KT > 8 ? 1 : (threads <= 160 ? 4 : (threads <= 288 ? 2 : 1)); }
+
+// Shared memory: full[4] empty[4] mbarriers, abort flag | rg[W][K] | S slots, each = item block + W rows of COLS*16 B.
+// The producer compacts on the way in: the r-th PRESENT worker's row lands in row r of the slot and its signed
+// weights in row r of the item block, so the compute threads index both by rank with constant strides.
+template <int KT, int COLS, int SPLIT>
+__global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 32))
+    decode_staged_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ DecodeTables tab,
+                         const __grid_constant__ StagedPlan plan) {
+  constexpr int KTP4 = ktp4(KT);
+  constexpr int NP = KTP4 / 2;                   // query pairs per thread
+  constexpr int kThreads = SPLIT * COLS;         // compute threads
+  constexpr int kConsumerWarps = kThreads / 32;
+  constexpr uint32_t kRowBytes = COLS * 16u;     // one worker's row inside a ring slot
+  constexpr int kWRowF = SPLIT * KTP4;           // floats of one rank's weights
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
+  uint64_t* empty = full + kMaxStages;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 64);
+  float* s_rg = reinterpret_cast<float*>(smem_raw + kTableOff);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int W = a.W, K = a.K, S = plan.stages;
+  const uint32_t wb = worker_bits(W);
+  const uint32_t Cv = (uint32_t)(a.C / 4);
+  unsigned char* slots = smem_raw + slots_off(W, K);
+  const uint32_t slot_sz = (uint32_t)slot_bytes(W, KT, SPLIT, COLS);
+  const uint32_t meta_sz = (uint32_t)meta_bytes(W, KT, SPLIT);
+  const bool producer = warp == kConsumerWarps;  // the last warp moves data and prepares items; the others compute
+  const bool literal = (a.flags & kFlagSignWorkerIndex) != 0;
+
+  const int KS = K | 1;  // odd row stride: a column of the table falls into distinct banks
+  for (int idx = tid; idx < W * K; idx += kThreads + 32) s_rg[(idx / K) * KS + idx % K] = tab.rg[idx];
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(smem_u32(full + s), 2);  // the copies' expect_tx arrival + the item block's arrival
+      mbar_init(smem_u32(empty + s), kConsumerWarps);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+
+  const int64_t first = blockIdx.x, stride = gridDim.x;
+  const int64_t my_items = first < plan.n_items ? (plan.n_items - first + stride - 1) / stride : 0;
+
+  // Bounded wait that also gives up when another warp of the CTA has given up.
+  auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+      if (mbar_try_wait(addr, parity)) return true;
+      if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    return false;
+  };
+  auto give_up = [&]() {
+    if (lane == 0) {
+      *abort_flag = 1;
+      atomicAdd(&g_decode_wait_timeouts, 1u);
+    }
+  };
+
+  if (producer) {
+    // This warp's work per item is a serial chain, so it is kept short: no 64-bit division (the item's group
+    // and tile advance incrementally), ranks from prefix population counts (lane = worker), conflict-free
+    // shared-memory traffic, and the masks of the next 32 items fetched together, one per lane, so that the
+    // latency of a global load is paid once per 32 items.
+    const int64_t dq = stride / plan.tiles;
+    const int32_t dr = (int32_t)(stride - dq * plan.tiles);
+    int64_t g = first / plan.tiles;
+    int32_t tile = (int32_t)(first - g * plan.tiles);
+    int64_t g_batch = g;  // group / tile of the first item of the next mask batch
+    int32_t tile_batch = tile;
+    uint32_t mask_batch = 0;
+    int64_t k = 0;
+    for (; k < my_items; ++k) {
+      if ((k & 31) == 0) {
+        // lane l fetches the mask of item k + l: its group is g_batch advanced l times
+        int64_t gl = g_batch + dq * lane;
+        const int64_t tl = (int64_t)tile_batch + (int64_t)dr * lane;
+        gl += tl / plan.tiles;
+        mask_batch = (k + lane < my_items) ? a.mask[gl] : 0u;
+        // advance the batch origin by 32 items
+        const int64_t t32 = (int64_t)tile_batch + (int64_t)dr * 32;
+        g_batch += dq * 32 + t32 / plan.tiles;
+        tile_batch = (int32_t)(t32 % plan.tiles);
+      }
+      const int stage = (int)(k % S);
+      if (k >= S && !wait(empty + stage, (uint32_t)(((k / S) - 1) & 1))) break;  // compute warps are done with the slot
+      const uint32_t col0 = (uint32_t)tile * COLS;
+      const uint32_t row_bytes = min((uint32_t)COLS, Cv - col0) * 16u;
+      unsigned char* mb = slots + (size_t)stage * slot_sz;
+      int32_t* hdr = reinterpret_cast<int32_t*>(mb);  // [0] = n
+      float* inv_den = reinterpret_cast<float*>(mb + 16);
+      float* w = reinterpret_cast<float*>(mb + kWeightsOff);
+      const uint32_t m = __shfl_sync(kFull, mask_batch, (int)(k & 31)) & wb;
+      const int n = __popc(m);
+      const bool present = (m >> lane) & 1u;               // lane = worker i
+      const int rank = __popc(m & ((1u << lane) - 1u));   // its position among the present workers
+      // 1. payload first, so that it is in flight while the item block is being written
+      const uint32_t bar = smem_u32(full + stage);
+      if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)n * row_bytes);
+      __syncwarp();
+      if (present) {
+        const float* src = a.Yt + g * a.y_gs + (int64_t)lane * a.y_rs + (int64_t)col0 * 4;
+        bulk_g2s(smem_u32(mb) + meta_sz + (uint32_t)rank * kRowBytes, src, row_bytes, bar);
+      }
+      // 2. signed weights by rank, lane = worker: w[rank][c] = +-rg[i][j(c)].  The column is rotated by the
+      //    lane so that the 32 stores of one step spread over the banks.
+      if (present) {
+        const bool neg = ((literal ? lane : rank) & 1) != 0;
+        const float* src = s_rg + lane * KS;
+        float* wr = w + rank * kWRowF;
+#pragma unroll
+        for (int c0 = 0; c0 < kWRowF; ++c0) {
+          const int c = (c0 + lane) % kWRowF;
+          const int h = c / KTP4, jj = c - h * KTP4;
+          const int j = h * KT + jj;
+          const float v = (jj < KT && j < K) ? src[j] : 0.f;
+          wr[c] = neg ? -v : v;
+        }
+      }
+      if (lane == 0) {
+        hdr[0] = n;
+        if (col0 == 0) {
+          if (a.n_used) a.n_used[g] = n;
+          if (a.status) a.status[g] = (n == 0 ? kStNoWorkers : 0u) | (n < K ? kStFewWorkers : 0u);
+        }
+      }
+      __syncwarp();
+      // 3. reciprocal denominators, lane = query j: the signed weights of query j summed in ascending worker
+      //    order, four loads at a time (rows beyond n contribute an exact 0)
+      {
+        float d = 0.f;
+        const int hq = lane / KT, jq = lane - hq * KT;
+        const float* wj = w + ((lane < K) ? hq * KTP4 + jq : 0);
+        for (int r0 = 0; r0 < n; r0 += 4) {
+          float t[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) t[u] = (r0 + u < n) ? wj[(r0 + u) * kWRowF] : 0.f;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) d += t[u];
+        }
+        inv_den[lane] = 1.0f / d;
+      }
+      __syncwarp();  // the whole item block is written before lane 0 publishes it
+      if (lane == 0) mbar_arrive(bar);
+      // next item of this CTA
+      g += dq;
+      tile += dr;
+      if (tile >= plan.tiles) {
+        tile -= plan.tiles;
+        ++g;
+      }
+    }
+    if (k < my_items) {
+      // A wait gave up (here or in a compute warp).  Let the copies already started land (bounded), then leave.
+      give_up();
+      for (int64_t q = (k > S ? k - S : 0); q < k; ++q) (void)mbar_wait(smem_u32(full + (q % S)), (uint32_t)((q / S) & 1));
+    }
+    return;
+  }
+
+  const int half = tid / COLS;
+  const uint32_t col = (uint32_t)(tid - half * COLS);
+
+  for (int64_t k = 0; k < my_items; ++k) {
+    const int stage = (int)(k % S);
+    if (!wait(full + stage, (uint32_t)((k / S) & 1))) {
+      give_up();
+      return;
+    }
+    const int64_t item = first + k * stride;
+    const int64_t g = item / plan.tiles;
+    const uint32_t col0 = (uint32_t)(item - g * plan.tiles) * COLS;
+    const uint32_t ncols = min((uint32_t)COLS, Cv - col0);
+    const unsigned char* mb = slots + (size_t)stage * slot_sz;
+    const int n = *reinterpret_cast<const int32_t*>(mb);
+    const float* inv_den = reinterpret_cast<const float*>(mb + 16);
+    // idle threads (beyond the last column) shadow column 0 and store nothing
+    const bool active = col < ncols;
+    const uint4* yp = reinterpret_cast<const uint4*>(mb + meta_sz) + (active ? col : 0u);               // + r * COLS
+    const ulonglong2* wp = reinterpret_cast<const ulonglong2*>(mb + kWeightsOff) + half * (KTP4 / 4);  // + r * kWRowF / 4
+
+    // acc[p][e] = (numerator of query 2p, numerator of query 2p+1) for payload element e of this column
+    uint64_t acc[NP][4];
+#pragma unroll
+    for (int p = 0; p < NP; ++p)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[p][e] = 0ull;
+
+    if (n > 0) {
+      // software pipeline over the ranks: the next row's payload and weights are loaded before this row's FMAs
+      uint4 yn = yp[0];
+      ulonglong2 wn[KTP4 / 4];
+#pragma unroll
+      for (int q = 0; q < KTP4 / 4; ++q) wn[q] = wp[q];
+#pragma unroll 2
+      for (int r = 0; r < n; ++r) {
+        const uint4 y = yn;
+        uint64_t wpair[NP];
+#pragma unroll
+        for (int q = 0; q < KTP4 / 4; ++q) {
+          wpair[2 * q] = wn[q].x;
+          wpair[2 * q + 1] = wn[q].y;
+        }
+        const int rn = min(r + 1, n - 1);
+        yn = yp[rn * COLS];
+#pragma unroll
+        for (int q = 0; q < KTP4 / 4; ++q) wn[q] = wp[rn * (kWRowF / 4) + q];
+        const uint64_t yd[4] = {dup(y.x), dup(y.y), dup(y.z), dup(y.w)};
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+          if (2 * p < KT) {  // pairs made only of padding are never touched
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[p][e] = ffma2(wpair[p], yd[e], acc[p][e]);
+          }
+        }
+      }
+    }
+
+    float inv[KT];
+#pragma unroll
+    for (int jj = 0; jj < KT; ++jj) inv[jj] = (half * KT + jj < K) ? inv_den[half * KT + jj] : 0.f;
+    // this warp no longer needs the slot
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(empty + stage));
+
+    float4* out = reinterpret_cast<float4*>(a.Yh + g * a.o_gs) + col0 + col;
+    const int64_t out_rs = a.o_rs / 4;
+#pragma unroll
+    for (int jj = 0; jj < KT; ++jj) {
+      const int j = half * KT + jj;
+      if (j < K && active) {
+        const int p = jj / 2;
+        float4 o;
+        if (jj & 1)
+          o = make_float4(inv[jj] * hi_f(acc[p][0]), inv[jj] * hi_f(acc[p][1]), inv[jj] * hi_f(acc[p][2]), inv[jj] * hi_f(acc[p][3]));
+        else
+          o = make_float4(inv[jj] * lo_f(acc[p][0]), inv[jj] * lo_f(acc[p][1]), inv[jj] * lo_f(acc[p][2]), inv[jj] * lo_f(acc[p][3]));
+        if (n == 0) o = make_float4(0.f, 0.f, 0.f, 0.f);
+        st_stream(out + j * out_rs, o);
+      }
+    }
+  }
+}
+
+int g_cfg_stages = 0;  // 0 = automatic; test / tuning hooks
+int g_cfg_ctas_per_sm = 0;
+int g_cfg_disable = 0;
+int g_cfg_cols = 0;
+int g_cfg_split = 0;
+
+template <int KT, int COLS, int SPLIT>
+cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream) {
+  const int64_t Cv = a.C / 4;
+  StagedPlan plan;
+  plan.tiles = (int32_t)((Cv + COLS - 1) / COLS);
+  plan.n_items = a.G * plan.tiles;
+  const int64_t slot = slot_bytes(a.W, KT, SPLIT, COLS);
+
+  int dev = 0, sms = 0, smem_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev)) != cudaSuccess) return e;
+  const int fixed = slots_off(a.W, a.K);
+  // as many CTAs per SM as fit with a two-slot ring (at most 4 small or 2 large ones), then the ring as deep
+  // as the rest allows
+  int ctas = min_ctas(KT, SPLIT * COLS + 32);
+  if (g_cfg_ctas_per_sm > 0 && g_cfg_ctas_per_sm < ctas) ctas = g_cfg_ctas_per_sm;
+  while (ctas > 1 && (int64_t)ctas * (fixed + 2 * slot + 1024) > smem_sm) --ctas;
+  int stages = (int)(((int64_t)smem_sm / ctas - 1024 - fixed) / slot);  // 1 KB per CTA is reserved
+  if (stages < 2) return cudaErrorInvalidConfiguration;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (g_cfg_stages >= 2 && g_cfg_stages < stages) stages = g_cfg_stages;
+  plan.stages = stages;
+  const size_t smem = (size_t)fixed + (size_t)stages * slot;
+  int64_t grid = (int64_t)sms * ctas;
+  if (grid > plan.n_items) grid = plan.n_items;
+
+  e = cudaFuncSetAttribute(decode_staged_kernel<KT, COLS, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  decode_staged_kernel<KT, COLS, SPLIT><<<(unsigned)grid, SPLIT * COLS + 32, smem, stream>>>(a, tab, plan);
+  count_launch();
+  return cudaGetLastError();
+}
+
+template <int SPLIT, int KT = 1>
+cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream) {
+  if constexpr (KT > kMaxK / SPLIT) {
+    return cudaErrorInvalidValue;
+  } else {
+    if (kt == KT) {
+      if (g_cfg_cols == 64) return launch_kt<KT, 64, SPLIT>(a, tab, stream);
+      return launch_kt<KT, 128, SPLIT>(a, tab, stream);
+    }
+    return dispatch_kt<SPLIT, KT + 1>(kt, a, tab, stream);
+  }
+}
+
+}  // namespace
+
+void decode_staged_config(int stages, int ctas_per_sm, int disable, int cols, int split) {
+  g_cfg_split = split;
+  g_cfg_stages = stages;
+  g_cfg_ctas_per_sm = ctas_per_sm;
+  g_cfg_disable = disable;
+  g_cfg_cols = cols;
+}
+
+// Wide rows on the 128-bit path.  Narrower payloads, and the (K, W) pairs in which some alpha_j equals some
+// beta_i (the row-copy case), stay on the register-staged kernel.
+bool decode_staged_eligible(const DecodeArgs& a) {
+  if (g_cfg_disable) return false;
+  const bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&
+                   a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  if (!(vec && a.C >= 512)) return false;
+  for (int j = 0; j < a.K; ++j)
+    for (int i = 0; i < a.W; ++i)
+      if (nodes_coincide(a.K, a.W, j, i)) return false;
+  return true;
+}
+
+cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream) {
+  if (g_cfg_split == 4) return dispatch_kt<4>((a.K + 3) / 4, a, tab, stream);
+  return dispatch_kt<2>((a.K + 1) / 2, a, tab, stream);
+}
+
+cudaError_t read_decode_wait_timeouts(unsigned int* out) {
+  return cudaMemcpyFromSymbol(out, g_decode_wait_timeouts, sizeof(unsigned int));
+}
+
+}  // namespace approxifer

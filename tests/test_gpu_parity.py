@@ -354,3 +354,65 @@ def test_strided_predictions_for_locate():
     adv, trusted = ap.approxifer_locate(ap.make_params(K, W, E), big.to(dev())[:, :, :C], ap.mask_tensor(mask))
     ref = oracle.locate(K, W, E, Yt.numpy(), mask)
     np.testing.assert_array_equal(adv.cpu().numpy(), ref["adv"])
+
+
+# ----------------------------------------------- wide-payload (staged) decoder
+
+STAGED_SHAPES = [
+    (16, 24, 300, 1000, 0),   # workload 4 shape: two column tiles per group (128 + 122 columns)
+    (12, 20, 37, 4000, 0),    # eight column tiles per group, ragged last tile
+    (8, 12, 200, 512, 0),     # smallest payload that takes the staged path
+    (3, 7, 60, 1024, 0),      # coincident nodes
+    (5, 9, 64, 2052, 1),      # literal sign: stays on the register-staged kernel
+    (32, 32, 9, 1028, 0),     # largest K and W
+    (7, 13, 50, 516, 0),      # odd K: the two halves own 4 and 3 queries
+    (1, 2, 20, 640, 0),       # K = 1: the second half of the CTA owns nothing
+]
+
+
+@pytest.mark.parametrize("stages,ctas,cols,split", [(0, 0, 0, 0), (2, 0, 128, 2), (3, 1, 128, 4), (4, 1, 64, 2), (2, 4, 64, 4), (0, 2, 64, 4)])
+def test_staged_decoder_matches_oracle_in_every_configuration(stages, ctas, cols, split):
+    try:
+        ap.debug_decode_config(stages, ctas, 0, cols, split)
+        for (K, W, G, C, flags) in STAGED_SHAPES:
+            rng = np.random.default_rng(C + K)
+            g = torch.Generator().manual_seed(C)
+            Yt = torch.randn((G, W, C), generator=g)
+            if flags == 0:
+                mask = random_masks(W, G, rng, min_present=0)
+                mask[0], mask[1], mask[2] = 2**W - 1, 0, 1 << (W - 1)
+            else:
+                mask = np.full(G, 2**W - 1, dtype=np.uint32)
+                mask[::3] = (2**W - 1) & ~1
+            dirty = Yt.clone()
+            for gi in range(G):
+                for i in range(W):
+                    if not (int(mask[gi]) >> i) & 1:
+                        dirty[gi, i] = float("nan")  # absent rows must never be used
+            n_used = torch.empty(G, dtype=torch.int32, device=dev())
+            status = torch.empty(G, dtype=torch.int32, device=dev())
+            out = torch.full((G, K, C + 4), CANARY, device=dev())
+            Yh = ap.approxifer_decode(ap.make_params(K, W, 0, flags), dirty.to(dev()), ap.mask_tensor(mask), out[:, :, :C],
+                                      n_used=n_used, status=status)
+            check_decode(K, W, Yt, mask, Yh, n_used, status, flags)
+            assert bool((out[:, :, C:] == CANARY).all())
+        assert ap.device_wait_timeouts() == 0
+    finally:
+        ap.debug_decode_config(0, 0, 0)
+
+
+def test_staged_and_register_decoders_agree_bitwise_on_sums_order():
+    """Both decoders add the same terms in the same order, so they agree to the last bit
+    except for the reciprocal-multiply of the denominator (identical too)."""
+    K, W, G, C = 12, 20, 64, 1000
+    rng = np.random.default_rng(1)
+    Yt = torch.randn((G, W, C), generator=torch.Generator().manual_seed(1)).to(dev())
+    mask = ap.mask_tensor(random_masks(W, G, rng, min_present=1))
+    p = ap.make_params(K, W)
+    a = ap.approxifer_decode(p, Yt, mask)
+    try:
+        ap.debug_decode_config(0, 0, 1)
+        b = ap.approxifer_decode(p, Yt, mask)
+    finally:
+        ap.debug_decode_config(0, 0, 0)
+    assert torch.equal(a, b)
