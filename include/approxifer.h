@@ -35,6 +35,7 @@
 #ifndef APPROXIFER_H_
 #define APPROXIFER_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -52,6 +53,7 @@ extern "C" {
 #define APPROXIFER_E_RANGE (-2) /* K not in 1..32, W not in 2..32, E < 0, G < 0, D < 1, D > 2^31, stride < row length */
 #define APPROXIFER_E_PARAM (-3) /* locate: E < 1 or 2(K+E) > W; unknown flag bits */
 #define APPROXIFER_E_CUDA (-4)  /* the CUDA runtime reported an error at launch */
+#define APPROXIFER_E_WORKSPACE (-5) /* host-buffer entry points: the device workspace cannot hold one group */
 
 /* params.flags */
 #define APPROXIFER_SIGN_RANK 0u         /* decoder sign (-1)^(rank of worker i among those used); default */
@@ -127,6 +129,32 @@ int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C,
                       const uint32_t* mask,
                       int32_t* adv, uint32_t* trusted_mask, uint32_t* status,
                       void* cuda_stream);
+
+/*
+ * Host-buffer variants of the three operations (same definitions and citations
+ * as above).  Payloads, masks and results live in HOST memory, dense
+ * ([G][K][D], [G][W][D], [G][W][C], [G][K][C], [G][E], [G]); pinned memory is
+ * needed for the copies to overlap.  `workspace` is caller-owned DEVICE memory
+ * of `workspace_bytes` bytes (256-byte aligned) used as staging; it is cut
+ * into one slice per stream, and the batch into chunks of whole groups that
+ * run as  copy in -> kernel -> copy out  on `cuda_streams[chunk % n_streams]`
+ * (an array of 1..8 cudaStream_t).  With two or more streams the transfers of
+ * neighbouring chunks overlap with each other and with the kernels.  The call
+ * only enqueues work: host and workspace buffers must stay untouched until
+ * every stream has been synchronised by the caller.  Nothing is allocated.
+ * APPROXIFER_E_WORKSPACE if a slice cannot hold a single group.
+ */
+int approxifer_encode_host(const approxifer_params* params, int64_t G, int64_t D,
+                           const float* hX, float* hXt,
+                           void* workspace, size_t workspace_bytes, void* const* cuda_streams, int n_streams);
+int approxifer_decode_host(const approxifer_params* params, int64_t G, int64_t C,
+                           const float* hYt, const uint32_t* hmask, float* hYhat,
+                           int32_t* hn_used /* or NULL */, uint32_t* hstatus /* or NULL */,
+                           void* workspace, size_t workspace_bytes, void* const* cuda_streams, int n_streams);
+int approxifer_locate_host(const approxifer_params* params, int64_t G, int64_t C,
+                           const float* hYt, const uint32_t* hmask,
+                           int32_t* hadv, uint32_t* htrusted_mask, uint32_t* hstatus /* or NULL */,
+                           void* workspace, size_t workspace_bytes, void* const* cuda_streams, int n_streams);
 
 /*
  * Test hook (not on the hot path): the weights the kernels use, computed on

@@ -10,6 +10,9 @@ from .binding import (  # noqa: F401
     approxifer_debug_weights,
     approxifer_decode,
     approxifer_encode,
+    approxifer_encode_host,
+    approxifer_decode_host,
+    approxifer_locate_host,
     approxifer_locate,
     approxifer_params,
     debug_decode_config,

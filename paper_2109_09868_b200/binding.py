@@ -18,7 +18,7 @@ import torch
 from . import build as _build
 
 OK = 0
-E_NULL, E_RANGE, E_PARAM, E_CUDA = -1, -2, -3, -4
+E_NULL, E_RANGE, E_PARAM, E_CUDA, E_WORKSPACE = -1, -2, -3, -4, -5
 SIGN_RANK, SIGN_WORKER_INDEX = 0, 1
 ST_NO_WORKERS, ST_FEW_WORKERS, ST_LOCATE_UNDERDETERMINED, ST_NONFINITE = 1, 2, 4, 8
 
@@ -32,6 +32,9 @@ EXPORTS = (
     "approxifer_launch_count",
     "approxifer_debug_decode_config",
     "approxifer_device_wait_timeouts",
+    "approxifer_encode_host",
+    "approxifer_decode_host",
+    "approxifer_locate_host",
 )
 
 
@@ -85,6 +88,15 @@ def load() -> ctypes.CDLL:
     lib.approxifer_debug_decode_config.argtypes = [c_int, c_int, c_int, c_int, c_int]
     lib.approxifer_debug_decode_config.restype = c_int
     lib.approxifer_device_wait_timeouts.restype = c_int64
+    c_size_t = ctypes.c_size_t
+    lib.approxifer_encode_host.argtypes = [pp, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, POINTER(c_void_p), c_int]
+    lib.approxifer_encode_host.restype = c_int
+    lib.approxifer_decode_host.argtypes = [pp, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                           c_size_t, POINTER(c_void_p), c_int]
+    lib.approxifer_decode_host.restype = c_int
+    lib.approxifer_locate_host.argtypes = [pp, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                           c_size_t, POINTER(c_void_p), c_int]
+    lib.approxifer_locate_host.restype = c_int
     del pf, pu, pi
     _lib = lib
     return lib
@@ -211,6 +223,66 @@ def approxifer_debug_weights(params: approxifer_params, mask: int = 0, which: in
         raise ApproxiferError(rc, "approxifer_debug_weights")
     nn = int(n.item())
     return w[:, :nn], idx[:nn]
+
+
+def _host(t: Optional[torch.Tensor], dtype, shape, name: str) -> int:
+    if t is None:
+        return 0
+    if t.is_cuda or t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous host %s tensor of shape %s" % (name, dtype, tuple(shape)))
+    return t.data_ptr()
+
+
+def _streams(streams):
+    arr = (c_void_p * len(streams))(*[int(s.cuda_stream) for s in streams])
+    return arr, len(streams)
+
+
+def _workspace(workspace: torch.Tensor):
+    if not workspace.is_cuda or not workspace.is_contiguous():
+        raise ValueError("workspace must be a contiguous CUDA tensor")
+    return workspace.data_ptr(), workspace.numel() * workspace.element_size()
+
+
+def approxifer_encode_host(params: approxifer_params, hX: torch.Tensor, hXt: torch.Tensor, workspace: torch.Tensor, streams) -> None:
+    """Host tensors hX [G][K][D] -> hXt [G][W][D], staged through the device `workspace` on `streams`.
+    Only enqueues; synchronise the streams before touching the buffers."""
+    G, K, D = hX.shape
+    wp, wbytes = _workspace(workspace)
+    arr, n = _streams(streams)
+    rc = load().approxifer_encode_host(ctypes.byref(params), G, D, _host(hX, torch.float32, (G, params.K, D), "hX"),
+                                       _host(hXt, torch.float32, (G, params.W, D), "hXt"), wp, wbytes, arr, n)
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_encode_host")
+
+
+def approxifer_decode_host(params: approxifer_params, hYt: torch.Tensor, hmask: torch.Tensor, hYhat: torch.Tensor,
+                           workspace: torch.Tensor, streams, hn_used: Optional[torch.Tensor] = None,
+                           hstatus: Optional[torch.Tensor] = None) -> None:
+    G, W, C = hYt.shape
+    wp, wbytes = _workspace(workspace)
+    arr, n = _streams(streams)
+    rc = load().approxifer_decode_host(ctypes.byref(params), G, C, _host(hYt, torch.float32, (G, params.W, C), "hYt"),
+                                       _host(hmask, torch.int32, (G,), "hmask"),
+                                       _host(hYhat, torch.float32, (G, params.K, C), "hYhat"),
+                                       _host(hn_used, torch.int32, (G,), "hn_used"), _host(hstatus, torch.int32, (G,), "hstatus"),
+                                       wp, wbytes, arr, n)
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_decode_host")
+
+
+def approxifer_locate_host(params: approxifer_params, hYt: torch.Tensor, hmask: torch.Tensor, hadv: torch.Tensor,
+                           htrusted: torch.Tensor, workspace: torch.Tensor, streams, hstatus: Optional[torch.Tensor] = None) -> None:
+    G, W, C = hYt.shape
+    wp, wbytes = _workspace(workspace)
+    arr, n = _streams(streams)
+    rc = load().approxifer_locate_host(ctypes.byref(params), G, C, _host(hYt, torch.float32, (G, params.W, C), "hYt"),
+                                       _host(hmask, torch.int32, (G,), "hmask"),
+                                       _host(hadv, torch.int32, (G, max(int(params.E), 0)), "hadv"),
+                                       _host(htrusted, torch.int32, (G,), "htrusted"), _host(hstatus, torch.int32, (G,), "hstatus"),
+                                       wp, wbytes, arr, n)
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_locate_host")
 
 
 def mask_tensor(mask_u32, device="cuda") -> torch.Tensor:

@@ -112,6 +112,7 @@ const char* approxifer_strerror(int code) {
     case APPROXIFER_E_RANGE: return "argument out of range (K in 1..32, W in 2..32, E >= 0, G >= 0, 1 <= D <= 2^31, row stride >= row length)";
     case APPROXIFER_E_PARAM: return "inconsistent parameters (locate needs E >= 1 and 2(K+E) <= W; unknown flag bits)";
     case APPROXIFER_E_CUDA: return "the CUDA runtime reported an error at kernel launch";
+    case APPROXIFER_E_WORKSPACE: return "the device workspace is too small to stage a single group";
     default: return "unknown error code";
   }
 }
