@@ -54,6 +54,7 @@ extern "C" {
 #define APPROXIFER_E_PARAM (-3) /* locate: E < 1 or 2(K+E) > W; unknown flag bits */
 #define APPROXIFER_E_CUDA (-4)  /* the CUDA runtime reported an error at launch */
 #define APPROXIFER_E_WORKSPACE (-5) /* host-buffer entry points: the device workspace cannot hold one group */
+#define APPROXIFER_E_TOO_LARGE (-6) /* approxifer_encode_host_static: the batch does not fit the built-in staging area */
 
 /* params.flags */
 #define APPROXIFER_SIGN_RANK 0u         /* decoder sign (-1)^(rank of worker i among those used); default */
@@ -155,6 +156,42 @@ int approxifer_locate_host(const approxifer_params* params, int64_t G, int64_t C
                            const float* hYt, const uint32_t* hmask,
                            int32_t* hadv, uint32_t* htrusted_mask, uint32_t* hstatus /* or NULL */,
                            void* workspace, size_t workspace_bytes, void* const* cuda_streams, int n_streams);
+
+/*
+ * Encoder for callers that cannot allocate device memory.  (The paper has no
+ * counterpart to this entry point; it computes exactly what approxifer_encode
+ * computes.)
+ *
+ * Who needs it: approxifer_encode_host wants a device workspace from its
+ * caller.  A front-end that shares the GPU with a model server which reserved
+ * all device memory at start-up has none to hand over, and a request path that
+ * must never call cudaMalloc (the call locks the device and synchronises it,
+ * stalling every other stream of the process) cannot create one.  Here the
+ * staging area is a fixed array of APPROXIFER_STATIC_WORKSPACE_BYTES bytes of
+ * device memory that is part of the library itself: every GPU the library is
+ * used on holds it from first use until the process exits.
+ *
+ *   hX   in,  HOST, dense [G][K][D]      hXt  out, HOST, dense [G][W][D]
+ *
+ * The whole batch is staged at once on `cuda_stream`: copy in, encode kernel,
+ * copy out; the call only enqueues and allocates nothing (no cudaMalloc, no
+ * cudaFree, no allocating library call).  With Dp = D rounded up to a multiple
+ * of 4, the batch must satisfy  4*G*Dp*(K+W) (+ up to 255 bytes of alignment)
+ * <= APPROXIFER_STATIC_WORKSPACE_BYTES, else APPROXIFER_E_TOO_LARGE is returned
+ * and nothing is enqueued.
+ *
+ * The first call on each device looks up the array's device address (one
+ * runtime query, no allocation); make that first call before starting any
+ * stream capture on that device.  All calls on a device share the one array,
+ * which keeps the previous call's bytes (nothing in it needs clearing: each
+ * call overwrites what it later reads).  Two calls whose GPU work can overlap
+ * -- different streams without an ordering between them, or several host
+ * threads -- race on the array and corrupt each other's results; order them on
+ * one stream or with events.
+ */
+#define APPROXIFER_STATIC_WORKSPACE_BYTES (32u << 20)
+int approxifer_encode_host_static(const approxifer_params* params, int64_t G, int64_t D,
+                                  const float* hX, float* hXt, void* cuda_stream);
 
 /*
  * Test hook (not on the hot path): the weights the kernels use, computed on

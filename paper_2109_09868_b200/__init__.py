@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     approxifer_decode,
     approxifer_encode,
     approxifer_encode_host,
+    approxifer_encode_host_static,
     approxifer_decode_host,
     approxifer_locate_host,
     approxifer_locate,

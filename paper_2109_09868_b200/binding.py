@@ -18,7 +18,8 @@ import torch
 from . import build as _build
 
 OK = 0
-E_NULL, E_RANGE, E_PARAM, E_CUDA, E_WORKSPACE = -1, -2, -3, -4, -5
+E_NULL, E_RANGE, E_PARAM, E_CUDA, E_WORKSPACE, E_TOO_LARGE = -1, -2, -3, -4, -5, -6
+STATIC_WORKSPACE_BYTES = 32 << 20
 SIGN_RANK, SIGN_WORKER_INDEX = 0, 1
 ST_NO_WORKERS, ST_FEW_WORKERS, ST_LOCATE_UNDERDETERMINED, ST_NONFINITE = 1, 2, 4, 8
 
@@ -35,6 +36,7 @@ EXPORTS = (
     "approxifer_encode_host",
     "approxifer_decode_host",
     "approxifer_locate_host",
+    "approxifer_encode_host_static",
 )
 
 
@@ -97,6 +99,8 @@ def load() -> ctypes.CDLL:
     lib.approxifer_locate_host.argtypes = [pp, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                            c_size_t, POINTER(c_void_p), c_int]
     lib.approxifer_locate_host.restype = c_int
+    lib.approxifer_encode_host_static.argtypes = [pp, c_int64, c_int64, c_void_p, c_void_p, c_void_p]
+    lib.approxifer_encode_host_static.restype = c_int
     del pf, pu, pi
     _lib = lib
     return lib
@@ -283,6 +287,17 @@ def approxifer_locate_host(params: approxifer_params, hYt: torch.Tensor, hmask: 
                                        wp, wbytes, arr, n)
     if rc != OK:
         raise ApproxiferError(rc, "approxifer_locate_host")
+
+
+def approxifer_encode_host_static(params: approxifer_params, hX: torch.Tensor, hXt: torch.Tensor, stream=None) -> None:
+    """Encoder for callers that cannot allocate device memory: host tensors hX [G][K][D] -> hXt [G][W][D],
+    staged through the library's built-in device array (at most STATIC_WORKSPACE_BYTES per call).  Only
+    enqueues on `stream`; synchronise it before reading hXt.  Calls that may overlap on the GPU race."""
+    G, K, D = hX.shape
+    rc = load().approxifer_encode_host_static(ctypes.byref(params), G, D, _host(hX, torch.float32, (G, params.K, D), "hX"),
+                                              _host(hXt, torch.float32, (G, params.W, D), "hXt"), _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_encode_host_static")
 
 
 def mask_tensor(mask_u32, device="cuda") -> torch.Tensor:

@@ -113,6 +113,7 @@ const char* approxifer_strerror(int code) {
     case APPROXIFER_E_PARAM: return "inconsistent parameters (locate needs E >= 1 and 2(K+E) <= W; unknown flag bits)";
     case APPROXIFER_E_CUDA: return "the CUDA runtime reported an error at kernel launch";
     case APPROXIFER_E_WORKSPACE: return "the device workspace is too small to stage a single group";
+    case APPROXIFER_E_TOO_LARGE: return "the batch is larger than the built-in staging area (APPROXIFER_STATIC_WORKSPACE_BYTES); split it or use approxifer_encode_host";
     default: return "unknown error code";
   }
 }

@@ -32,7 +32,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_version_and_strerror():
     assert ap.version() == 100
-    for code in (0, -1, -2, -3, -4, -5):
+    for code in (0, -1, -2, -3, -4, -5, -6):
         assert ap.strerror(code) and "unknown error" not in ap.strerror(code)
     assert "unknown error" in ap.strerror(-99)
 
