@@ -38,6 +38,10 @@ UNIT = "GB/s"
 HEADLINE_CFG = 2
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
+# DRAM traffic of encode_kernel<8, float4> per group of the headline workload, from the ncu capture of a
+# 4096-group launch: (402.663 MB read + 546.9 MB written) / 4096.  Traffic is proportional to the number
+# of groups (every row is touched once); the written part misses the dirty lines still in L2 at kernel end.
+ENCODE_TRAFFIC_PER_GROUP = (402.663e6 + 546.9e6) / 4096
 
 
 # ----------------------------------------------------------------- byte counts
@@ -498,7 +502,8 @@ def main():
         "kernels": {"encode_ms": enc_ms, "encode_GB_per_s": enc_gbs, "decode_ms": dec_ms,
                     "decode_GB_per_s": dec_b / dec_ms / 1e6, "decode_groups_per_s": w.G / dec_ms * 1e3},
         "roofline": {"bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": enc_gbs / peak, "peak_source": peak_src, "traffic": None,
+                     "frac": enc_gbs / peak, "peak_source": peak_src, "traffic": ENCODE_TRAFFIC_PER_GROUP * w.G,
+                     "traffic_source": "ncu dram read+write bytes of a 4096-group launch of the unchanged kernel, per group x groups",
                      "algorithmic_bytes_per_launch": enc_b},
         "clocks": clocks,
         "gpu_launches": launches,
