@@ -17,6 +17,11 @@
 // memory) and needs no cross-lane reduction.  floor(32/m) classes (at most 8)
 // are factorised side by side in one warp.  The selection steps (E smallest
 // |a_r|, E most voted) are warp arg-min / arg-max butterflies with lane = worker.
+//
+// The kernel is compiled per (NMAX, M): NMAX = rows rounded up to 8, M = K+E.
+// With M fixed at compile time every loop over rows and columns has static
+// bounds: reflector k of the P-block touches rows k.., reflector k of the
+// reduced problem rows M+k.., and no element is masked by a run-time predicate.
 #include "common.cuh"
 
 namespace approxifer {
@@ -28,16 +33,16 @@ constexpr int kLocateThreads = kLocateWarps * 32;
 constexpr int kMaxSlots = 8;
 constexpr unsigned kFull = 0xffffffffu;
 
-template <int NMAX>
+template <int NMAX, int M>
 struct WarpSmem {
-  static constexpr int MMAX = NMAX / 2;
-  double refl[MMAX][NMAX];          // normalised reflectors of the P-block (H = I - v v^T)
-  double pw[NMAX][MMAX];            // pw[r][k] = b_r^k
-  double vbuf[2][kMaxSlots][NMAX];  // reflector being broadcast, per class slot, double-buffered
-  double rs[32][MMAX];              // rs[lane][k'] = row k' of that lane's column of the reduced R | rhs
-  double qs[32];                    // Q_1.. of each slot
-  double xs[NMAX];                  // b_r
-  long long yoff[NMAX];             // element offset of worker F[r]'s row
+  static constexpr int kSlots = (32 / M) < kMaxSlots ? (32 / M) : kMaxSlots;
+  double refl[M][NMAX];            // normalised reflectors of the P-block (H = I - v v^T)
+  double pw[NMAX][M];              // pw[r][k] = b_r^k
+  double vbuf[2][kSlots][NMAX];    // reflector being broadcast, per class slot, double-buffered
+  double rs[32][M];                // rs[lane][k'] = row k' of that lane's column of the reduced R | rhs
+  double qs[32];                   // Q_1.. of each slot
+  double xs[NMAX];                 // b_r
+  long long yoff[NMAX];            // element offset of worker F[r]'s row
 };
 
 // Lexicographic "smaller (key, index)" butterfly: returns the index of the
@@ -55,64 +60,97 @@ __device__ __forceinline__ int warp_argmin(double key, int idx) {
   return idx;
 }
 
-// Builds the normalised reflector of `col` restricted to rows >= row0:
-// v = x - akk e_row0 scaled so that H = I - v v^T maps x to akk e_row0.
-// Returns akk (0 and v = 0 when the sub-column is exactly zero).
-template <int NMAX>
-__device__ __forceinline__ double make_reflector(const double (&col)[NMAX], int row0, double* v_out) {
-  double s2 = 0.0, x0 = 0.0;
+// Normalised reflector of `col` restricted to rows >= ROW0:
+// v = (x - akk e_ROW0) / sqrt(c), c = |x|(|x| + |x_ROW0|), so that H = I - v v^T
+// maps x to akk e_ROW0.  v_out[r] is written for r >= (ROW0 rounded down to even);
+// returns akk (0 and v = 0 when the sub-column is exactly zero).
+template <int NMAX, int ROW0>
+__device__ __forceinline__ double make_reflector(const double (&col)[NMAX], double* v_out) {
+  double s2a = 0.0, s2b = 0.0;
 #pragma unroll
-  for (int r = 0; r < NMAX; ++r) {
-    const double x = (r >= row0) ? col[r] : 0.0;
-    s2 = fma(x, x, s2);
-    x0 = (r == row0) ? col[r] : x0;
+  for (int r = ROW0; r < NMAX; r += 2) {
+    s2a = fma(col[r], col[r], s2a);
+    if (r + 1 < NMAX) s2b = fma(col[r + 1], col[r + 1], s2b);
   }
-  const double normx = sqrt(s2);
+  const double s2 = s2a + s2b;
+  const double x0 = col[ROW0];
+  const bool nz = s2 > 0.0;
+  const double normx = nz ? s2 * rsqrt(s2) : 0.0;
   const double akk = (x0 >= 0.0) ? -normx : normx;
-  // v^T v = s2 - x0^2 + (x0 - akk)^2 = 2 (s2 - x0 akk) = 2 normx (normx + |x0|)
-  const double vv = 2.0 * (s2 - x0 * akk);
-  const double scale = (vv > 0.0) ? sqrt(2.0 / vv) : 0.0;
+  const double c = fma(fabs(x0), normx, s2);
+  const double scale = nz ? rsqrt(c) : 0.0;
+  if (ROW0 & 1) v_out[ROW0 - 1] = 0.0;
+  v_out[ROW0] = (x0 - akk) * scale;
 #pragma unroll
-  for (int r = 0; r < NMAX; ++r) {
-    double v = (r > row0) ? col[r] : 0.0;
-    v = (r == row0) ? (x0 - akk) : v;
-    v_out[r] = v * scale;
-  }
-  return (vv > 0.0) ? akk : 0.0;
+  for (int r = ROW0 + 1; r < NMAX; ++r) v_out[r] = col[r] * scale;
+  return akk;
 }
 
-template <int NMAX>
+// col <- (I - v v^T) col for a reflector whose entries before ROW0 are zero.
+template <int NMAX, int ROW0>
 __device__ __forceinline__ void apply_reflector(double (&col)[NMAX], const double* v) {
-  double s = 0.0;
+  constexpr int R0 = ROW0 & ~1;
+  double2 vv[(NMAX - R0) / 2];
+  double sa = 0.0, sb = 0.0;
 #pragma unroll
-  for (int r = 0; r < NMAX; r += 2) {
-    const double2 vv = *reinterpret_cast<const double2*>(v + r);
-    s = fma(vv.x, col[r], s);
-    s = fma(vv.y, col[r + 1], s);
+  for (int r = R0; r < NMAX; r += 2) {
+    vv[(r - R0) / 2] = *reinterpret_cast<const double2*>(v + r);
+    sa = fma(vv[(r - R0) / 2].x, col[r], sa);
+    sb = fma(vv[(r - R0) / 2].y, col[r + 1], sb);
   }
+  const double s = -(sa + sb);
 #pragma unroll
-  for (int r = 0; r < NMAX; r += 2) {
-    const double2 vv = *reinterpret_cast<const double2*>(v + r);
-    col[r] = fma(-s, vv.x, col[r]);
-    col[r + 1] = fma(-s, vv.y, col[r + 1]);
+  for (int r = R0; r < NMAX; r += 2) {
+    col[r] = fma(s, vv[(r - R0) / 2].x, col[r]);
+    col[r + 1] = fma(s, vv[(r - R0) / 2].y, col[r + 1]);
   }
 }
 
-template <int NMAX>
+// Compile-time loops over reflector indices.
+template <int NMAX, int M, int K0 = 0>
+__device__ __forceinline__ void pblock_factor(double (&col)[NMAX], int lane, WarpSmem<NMAX, M>& sm) {
+  if constexpr (K0 < M) {
+    if (lane == K0) make_reflector<NMAX, K0>(col, sm.refl[K0]);
+    __syncwarp();
+    if (lane > K0 && lane < M) apply_reflector<NMAX, K0>(col, sm.refl[K0]);
+    pblock_factor<NMAX, M, K0 + 1>(col, lane, sm);
+  }
+}
+template <int NMAX, int M, int K0 = 0>
+__device__ __forceinline__ void pblock_apply(double (&col)[NMAX], const WarpSmem<NMAX, M>& sm) {
+  if constexpr (K0 < M) {
+    apply_reflector<NMAX, K0>(col, sm.refl[K0]);
+    pblock_apply<NMAX, M, K0 + 1>(col, sm);
+  }
+}
+template <int NMAX, int M, int K0 = 0>
+__device__ __forceinline__ void reduced_factor(double (&col)[NMAX], bool active, int l, int slot, double& diag,
+                                               WarpSmem<NMAX, M>& sm) {
+  if constexpr (K0 < M - 1) {
+    double* vb = sm.vbuf[K0 & 1][slot];
+    if (active && l == K0) diag = make_reflector<NMAX, M + K0>(col, vb);
+    __syncwarp();
+    if (active && l > K0) apply_reflector<NMAX, M + K0>(col, vb);
+    reduced_factor<NMAX, M, K0 + 1>(col, active, l, slot, diag, sm);
+  }
+}
+
+template <int NMAX, int M>
 __global__ void __launch_bounds__(kLocateThreads) locate_kernel(const __grid_constant__ LocateArgs a,
                                                                 const __grid_constant__ LocateTables tab) {
-  constexpr int MMAX = NMAX / 2;
+  using SM = WarpSmem<NMAX, M>;
+  constexpr int kSlots = SM::kSlots;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  WarpSmem<NMAX>& sm = reinterpret_cast<WarpSmem<NMAX>*>(smem_raw)[warp];
+  SM& sm = reinterpret_cast<SM*>(smem_raw)[warp];
 
   const int64_t g = (int64_t)blockIdx.x * kLocateWarps + warp;
   if (g >= a.G) return;  // whole warp leaves together
 
-  const int E = a.E, m = a.K + E;
+  const int E = a.E;
   const uint32_t mask = a.mask[g] & worker_bits(a.W);
   const int n = __popc(mask);
-  if (n < 2 * m) {  // Algorithm 1's condition N-S+1 >= 2(K+E) does not hold
+  if (n < 2 * M) {  // Algorithm 1's condition N-S+1 >= 2(K+E) does not hold
     for (int e = lane; e < E; e += 32) a.adv[g * E + e] = -1;
     if (lane == 0) {
       a.trusted[g] = mask;
@@ -128,7 +166,8 @@ __global__ void __launch_bounds__(kLocateThreads) locate_kernel(const __grid_con
     sm.xs[lane] = b;
     sm.yoff[lane] = (lane < n) ? (long long)my_worker * a.y_rs : 0;
     double p = 1.0;
-    for (int k = 0; k < m; ++k) {
+#pragma unroll
+    for (int k = 0; k < M; ++k) {
       sm.pw[lane][k] = (lane < n) ? p : 0.0;
       p *= b;
     }
@@ -137,88 +176,77 @@ __global__ void __launch_bounds__(kLocateThreads) locate_kernel(const __grid_con
 
   // ---- P-block: Householder reflectors of V = [b_r^k], lane = column k --------
   double col[NMAX];
-  {
 #pragma unroll
-    for (int r = 0; r < NMAX; ++r) col[r] = (lane < m) ? sm.pw[r][lane] : 0.0;
-    for (int k = 0; k < m; ++k) {
-      if (lane == k) make_reflector<NMAX>(col, k, sm.refl[k]);
-      __syncwarp();
-      if (lane > k && lane < m) apply_reflector<NMAX>(col, sm.refl[k]);
-    }
-  }
+  for (int r = 0; r < NMAX; ++r) col[r] = (lane < M) ? sm.pw[r][lane] : 0.0;
+  pblock_factor<NMAX, M>(col, lane, sm);
   __syncwarp();
 
-  // ---- classes, `slots` at a time; lane = (slot, column l) ---------------------
-  int slots = 32 / m;
-  if (slots > kMaxSlots) slots = kMaxSlots;
-  const int slot = lane / m, l = lane - slot * m;
-  const bool lane_in_slot = slot < slots;
+  // ---- classes, kSlots at a time; lane = (slot, column l) ----------------------
+  const int slot_raw = lane / M, l = lane - slot_raw * M;
+  const bool lane_in_slot = slot_raw < kSlots;
+  const int slot = lane_in_slot ? slot_raw : 0;
   const float* Yg = a.Yt + g * a.y_gs;
 
-  int votes = 0;       // lane = worker r again: how often it was among the E smallest
+  int votes = 0;  // lane = worker r again: how often it was among the E smallest
   uint32_t st = 0;
 
-  for (int64_t c0 = 0; c0 < a.C; c0 += slots) {
-    const int64_t c = c0 + slot;
+  for (int64_t c0 = 0; c0 < a.C; c0 += kSlots) {
+    const int64_t c = c0 + slot_raw;
     const bool active = lane_in_slot && c < a.C;
 
-    // column l < m-1: -y_r b_r^(l+1);  column m-1: the right-hand side y_r
+    // column l < M-1: -y_r b_r^(l+1);  column M-1: the right-hand side y_r  (rows >= n are zero)
+    {
+      const int lp = (l < M - 1) ? l + 1 : 0;
+      const double sgn = (l < M - 1) ? -1.0 : 1.0;  // pw[r][0] = 1 on present rows
 #pragma unroll
-    for (int r = 0; r < NMAX; ++r) {
-      double v = 0.0;
-      if (active && r < n) {
-        const double y = (double)__ldg(Yg + sm.yoff[r] + c);
-        v = (l < m - 1) ? -y * sm.pw[r][l + 1] : y;
+      for (int r = 0; r < NMAX; ++r) {
+        double v = 0.0;
+        if (active && r < n) v = sgn * (double)__ldg(Yg + sm.yoff[r] + c) * sm.pw[r][lp];
+        col[r] = v;
       }
-      col[r] = v;
     }
-    // eliminate P: apply H_0 .. H_{m-1}
-    for (int k = 0; k < m; ++k) apply_reflector<NMAX>(col, sm.refl[k]);
+    // eliminate P: apply H_0 .. H_{M-1}
+    pblock_apply<NMAX, M>(col, sm);
 
-    // reduced problem on rows m..n-1: Householder QR, one column per step
+    // reduced problem on rows M..n-1: Householder QR, one column per step
     double diag = 0.0;
-    for (int k = 0; k < m - 1; ++k) {
-      double* vb = sm.vbuf[k & 1][lane_in_slot ? slot : 0];
-      if (active && l == k) diag = make_reflector<NMAX>(col, m + k, vb);
-      __syncwarp();
-      if (active && l > k) apply_reflector<NMAX>(col, vb);
-    }
-    // R (upper triangle, rows m..2m-2 of the columns) and rhs -> shared memory
+    reduced_factor<NMAX, M>(col, active, l, slot, diag, sm);
+
+    // R (upper triangle, rows M..2M-2 of the columns) and rhs -> shared memory
     if (active) {
 #pragma unroll
-      for (int r = 0; r < NMAX; ++r)
-        if (r >= m && r < 2 * m - 1) sm.rs[lane][r - m] = col[r];
+      for (int r = M; r < 2 * M - 1; ++r) sm.rs[lane][r - M] = col[r];
     }
     __syncwarp();
 
-    // back substitution, lane = (slot, row l) for l < m-1
-    {
-      double rhs = 0.0, rrow[MMAX];
-      const int base = slot * m;
+    // back substitution, lane = (slot, row l) for l < M-1
+    if constexpr (M > 1) {
+      double rhs = 0.0, rrow[M - 1];
+      const int base = slot * M;
+      const bool row_lane = active && l < M - 1;
 #pragma unroll
-      for (int k = 0; k < MMAX; ++k) rrow[k] = (active && k < m - 1 && l < m - 1) ? sm.rs[base + k][l] : 0.0;
-      if (active && l < m - 1) rhs = sm.rs[base + m - 1][l];
+      for (int k = 0; k < M - 1; ++k) rrow[k] = row_lane ? sm.rs[base + k][l] : 0.0;
+      if (row_lane) rhs = sm.rs[base + M - 1][l];
       const double invd = (diag != 0.0) ? 1.0 / diag : 0.0;  // a zero column leaves its unknown at 0
 #pragma unroll
-      for (int k = MMAX - 2; k >= 0; --k) {
-        if (k < m - 1) {
-          const int src = lane_in_slot ? base + k : lane;
-          const double qk = __shfl_sync(kFull, rhs * invd, src);
-          if (l < k) rhs = fma(-rrow[k], qk, rhs);
-        }
+      for (int k = M - 2; k >= 0; --k) {
+        const int src = lane_in_slot ? base + k : lane;
+        const double qk = __shfl_sync(kFull, rhs * invd, src);
+        if (l < k) rhs = fma(-rrow[k], qk, rhs);
       }
-      if (active && l < m - 1) sm.qs[lane] = rhs * invd;
+      if (row_lane) sm.qs[lane] = rhs * invd;
     }
     __syncwarp();
 
     // a_r = Q(b_r) = 1 + sum_{k>=1} Q_k b_r^k, lane = worker r; then the E smallest |a_r|
-    for (int s = 0; s < slots && c0 + s < a.C; ++s) {
+    for (int s = 0; s < kSlots && c0 + s < a.C; ++s) {
       double mag = INFINITY;
       if (lane < n) {
         const double b = sm.xs[lane];
         double q = 1.0, p = b;
-        for (int k = 0; k < m - 1; ++k) {
-          q = fma(sm.qs[s * m + k], p, q);
+#pragma unroll
+        for (int k = 0; k < M - 1; ++k) {
+          q = fma(sm.qs[s * M + k], p, q);
           p *= b;
         }
         mag = fabs(q);
@@ -268,18 +296,29 @@ __global__ void __launch_bounds__(kLocateThreads) locate_kernel(const __grid_con
   }
 }
 
-template <int NMAX>
-cudaError_t launch_n(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream) {
-  const size_t smem = sizeof(WarpSmem<NMAX>) * kLocateWarps;
+template <int NMAX, int M>
+cudaError_t launch_nm(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream) {
+  const size_t smem = sizeof(WarpSmem<NMAX, M>) * kLocateWarps;
   if (smem > 48 * 1024) {  // opt in to more than the default dynamic shared memory (per device, idempotent)
-    cudaError_t e = cudaFuncSetAttribute(locate_kernel<NMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(locate_kernel<NMAX, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   const int64_t blocks = (a.G + kLocateWarps - 1) / kLocateWarps;
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-  locate_kernel<NMAX><<<(unsigned)blocks, kLocateThreads, smem, stream>>>(a, tab);
+  locate_kernel<NMAX, M><<<(unsigned)blocks, kLocateThreads, smem, stream>>>(a, tab);
   count_launch();
   return cudaGetLastError();
+}
+
+// m = K + E runs over 2 .. NMAX/2 (the entry point has checked 2m <= W <= NMAX).
+template <int NMAX, int M = 2>
+cudaError_t dispatch_m(int m, const LocateArgs& a, const LocateTables& tab, cudaStream_t stream) {
+  if constexpr (M > NMAX / 2) {
+    return cudaErrorInvalidValue;
+  } else {
+    if (m == M) return launch_nm<NMAX, M>(a, tab, stream);
+    return dispatch_m<NMAX, M + 1>(m, a, tab, stream);
+  }
 }
 
 }  // namespace
@@ -288,10 +327,11 @@ cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   LocateTables tab;
   build_locate_tables(a.W, &tab);
-  if (a.W <= 8) return launch_n<8>(a, tab, stream);
-  if (a.W <= 16) return launch_n<16>(a, tab, stream);
-  if (a.W <= 24) return launch_n<24>(a, tab, stream);
-  return launch_n<32>(a, tab, stream);
+  const int m = a.K + a.E;
+  if (a.W <= 8) return dispatch_m<8>(m, a, tab, stream);
+  if (a.W <= 16) return dispatch_m<16>(m, a, tab, stream);
+  if (a.W <= 24) return dispatch_m<24>(m, a, tab, stream);
+  return dispatch_m<32>(m, a, tab, stream);
 }
 
 }  // namespace approxifer
