@@ -290,8 +290,16 @@ def other_workloads(ap, dev, peak):
     Yh = torch.empty((w5.G, w5.K, w5.C), device=dev)
     med, mn = time_launches(lambda: ap.approxifer_locate(p5, Yt, mt, adv, trusted), 3, 10)
     recall = float((adv.cpu().numpy() == adv_true).all(axis=1).mean())
+    # Algorithm 2 as printed: per class a least-squares problem with n rows and m' = 2(K+E)-1 unknowns,
+    # 2 n m'^2 - (2/3) m'^3 flop by Householder QR; fp64 peak = 64 FMA lanes/SM/clock.
+    n5, mp5 = w5.W - w5.S, 2 * (w5.K + w5.E) - 1
+    flops = w5.G * w5.C * (2.0 * n5 * mp5 * mp5 - (2.0 / 3.0) * mp5 ** 3)
+    fp64_peak = 148 * 64 * 2 * 1.965e9 / 1e12
     entry("configs[4] locate K=8 W=24 E=2 C=10 (fp64 solve, ALU-bound; L2-resident input)", locate_bytes(w5, m5), med, mn, w5.G,
-          {"located_equals_injected": recall})
+          {"located_equals_injected": recall,
+           "roofline": {"bound": "alu", "achieved": flops / med / 1e9, "peak": fp64_peak, "unit": "TFLOP/s",
+                        "frac": flops / med / 1e9 / fp64_peak,
+                        "note": "algorithmic fp64 flop of Algorithm 2's per-class least squares / time; peak = 148 SMs x 64 DFMA/clk x 2 x 1.965 GHz"}})
     t5 = trusted.cpu().numpy().view(np.uint32)
     med, mn = time_launches(lambda: ap.approxifer_decode(p5, Yt, trusted, Yh), 3, 10)
     entry("configs[4] decode from trusted K=8 W=24 C=10 (L2-resident)", decode_bytes(w5, t5), med, mn, w5.G)
