@@ -416,3 +416,20 @@ def test_staged_and_register_decoders_agree_bitwise_on_sums_order():
     finally:
         ap.debug_decode_config(0, 0, 0)
     assert torch.equal(a, b)
+
+
+def test_worker_major_layouts_for_decode_and_locate():
+    """Coded predictions stored per worker ([W][G][C], the layout in which the workers' answers arrive) are
+    addressed through the strides; both decoders and the locator must accept them."""
+    K, E, S, W, G = 8, 2, 2, 24, 64
+    for C in (10, 1000):
+        Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=C)
+        wm = Yt.permute(1, 0, 2).contiguous().to(dev())          # [W][G][C]
+        view = wm.permute(1, 0, 2)                                # [G][W][C] view: gstride = C, rstride = G*C
+        p = ap.make_params(K, W, E)
+        adv, trusted = ap.approxifer_locate(p, view, ap.mask_tensor(mask))
+        ref = oracle.locate(K, W, E, Yt.numpy(), mask)
+        np.testing.assert_array_equal(adv.cpu().numpy(), ref["adv"])
+        out = torch.empty((K, G, C), device=dev())               # query-major output
+        ap.approxifer_decode(p, view, trusted, out.permute(1, 0, 2))
+        check_decode(K, W, Yt, ref["trusted"], out.permute(1, 0, 2))
