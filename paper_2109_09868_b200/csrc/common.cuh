@@ -60,6 +60,11 @@ cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, c
 void decode_staged_config(int stages, int ctas_per_sm, int disable, int cols, int split);
 cudaError_t read_decode_wait_timeouts(unsigned int* out);
 
+// Thread-per-class locator for K+E <= kLocateRowsMaxM (locate_rows.cu); the warp-per-group kernel covers the rest.
+constexpr int kLocateRowsMaxM = 10;
+cudaError_t launch_locate_rows(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream);
+void locate_config(int force_warp_kernel);
+
 void count_launch(int n = 1);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

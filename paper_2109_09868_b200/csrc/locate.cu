@@ -23,15 +23,17 @@
 // bounds: reflector k of the P-block touches rows k.., reflector k of the
 // reduced problem rows M+k.., and no element is masked by a run-time predicate.
 #include "common.cuh"
+#include "locate_common.cuh"
 
 namespace approxifer {
 
 namespace {
 
+using namespace locate_detail;
+
 constexpr int kLocateWarps = 4;
 constexpr int kLocateThreads = kLocateWarps * 32;
 constexpr int kMaxSlots = 8;
-constexpr unsigned kFull = 0xffffffffu;
 
 template <int NMAX, int M>
 struct WarpSmem {
@@ -44,67 +46,6 @@ struct WarpSmem {
   double xs[NMAX];                 // b_r
   long long yoff[NMAX];            // element offset of worker F[r]'s row
 };
-
-// Lexicographic "smaller (key, index)" butterfly: returns the index of the
-// minimum over the warp; ties go to the lower index.
-__device__ __forceinline__ int warp_argmin(double key, int idx) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const double k2 = __shfl_xor_sync(kFull, key, o);
-    const int i2 = __shfl_xor_sync(kFull, idx, o);
-    if (k2 < key || (k2 == key && i2 < idx)) {
-      key = k2;
-      idx = i2;
-    }
-  }
-  return idx;
-}
-
-// Normalised reflector of `col` restricted to rows >= ROW0:
-// v = (x - akk e_ROW0) / sqrt(c), c = |x|(|x| + |x_ROW0|), so that H = I - v v^T
-// maps x to akk e_ROW0.  v_out[r] is written for r >= (ROW0 rounded down to even);
-// returns akk (0 and v = 0 when the sub-column is exactly zero).
-template <int NMAX, int ROW0>
-__device__ __forceinline__ double make_reflector(const double (&col)[NMAX], double* v_out) {
-  double s2a = 0.0, s2b = 0.0;
-#pragma unroll
-  for (int r = ROW0; r < NMAX; r += 2) {
-    s2a = fma(col[r], col[r], s2a);
-    if (r + 1 < NMAX) s2b = fma(col[r + 1], col[r + 1], s2b);
-  }
-  const double s2 = s2a + s2b;
-  const double x0 = col[ROW0];
-  const bool nz = s2 > 0.0;
-  const double normx = nz ? s2 * rsqrt(s2) : 0.0;
-  const double akk = (x0 >= 0.0) ? -normx : normx;
-  const double c = fma(fabs(x0), normx, s2);
-  const double scale = nz ? rsqrt(c) : 0.0;
-  if (ROW0 & 1) v_out[ROW0 - 1] = 0.0;
-  v_out[ROW0] = (x0 - akk) * scale;
-#pragma unroll
-  for (int r = ROW0 + 1; r < NMAX; ++r) v_out[r] = col[r] * scale;
-  return akk;
-}
-
-// col <- (I - v v^T) col for a reflector whose entries before ROW0 are zero.
-template <int NMAX, int ROW0>
-__device__ __forceinline__ void apply_reflector(double (&col)[NMAX], const double* v) {
-  constexpr int R0 = ROW0 & ~1;
-  double2 vv[(NMAX - R0) / 2];
-  double sa = 0.0, sb = 0.0;
-#pragma unroll
-  for (int r = R0; r < NMAX; r += 2) {
-    vv[(r - R0) / 2] = *reinterpret_cast<const double2*>(v + r);
-    sa = fma(vv[(r - R0) / 2].x, col[r], sa);
-    sb = fma(vv[(r - R0) / 2].y, col[r + 1], sb);
-  }
-  const double s = -(sa + sb);
-#pragma unroll
-  for (int r = R0; r < NMAX; r += 2) {
-    col[r] = fma(s, vv[(r - R0) / 2].x, col[r]);
-    col[r + 1] = fma(s, vv[(r - R0) / 2].y, col[r + 1]);
-  }
-}
 
 // Compile-time loops over reflector indices.
 template <int NMAX, int M, int K0 = 0>
@@ -321,13 +262,18 @@ cudaError_t dispatch_m(int m, const LocateArgs& a, const LocateTables& tab, cuda
   }
 }
 
+int g_force_warp_kernel = 0;  // test hook
+
 }  // namespace
+
+void locate_config(int force_warp_kernel) { g_force_warp_kernel = force_warp_kernel; }
 
 cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   LocateTables tab;
   build_locate_tables(a.W, &tab);
   const int m = a.K + a.E;
+  if (m <= kLocateRowsMaxM && !g_force_warp_kernel) return launch_locate_rows(a, tab, stream);
   if (a.W <= 8) return dispatch_m<8>(m, a, tab, stream);
   if (a.W <= 16) return dispatch_m<16>(m, a, tab, stream);
   if (a.W <= 24) return dispatch_m<24>(m, a, tab, stream);

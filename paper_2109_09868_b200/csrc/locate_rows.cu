@@ -1,0 +1,321 @@
+// ApproxIFER Byzantine-worker locator (Algorithm 2), thread-per-class variant for K+E <= 10.
+//
+// Same mathematics as locate_kernel (locate.cu): the P-part of the per-class least-squares problem is
+// eliminated with an orthonormal basis N of the complement of {polynomials of degree < M} on the available
+// nodes (M = K+E), which depends on the mask only, and the Q-part solves the (n-M) x (M-1) problem
+//     B q = -b0,   B[r][l] = sum_i N[i][r] y_i b_i^l (l = 1..M-1),   b0[r] = sum_i N[i][r] y_i.
+// Different parallelisation: after one warp per group has produced N (Householder reflectors of the
+// Vandermonde block applied to unit vectors, lane = column), every (group, class) pair gets ONE THREAD.
+// The thread generates the rows of [B | -b0] one at a time from N (shared memory, shared by the group's
+// threads) and its own 22-odd predictions (registers) and folds each row into an upper-triangular factor
+// with Givens rotations.  The factor (at most 45 + 9 doubles) lives in registers with static indices; the
+// rows are never stored.  No lane waits for another lane: there is no serial single-lane section, and all
+// 32 lanes of a warp work on different problems.  The thread then evaluates a_r = Q(b_r) for every
+// available worker, picks the E smallest |a_r| (ties to the lower worker) and votes with shared-memory
+// atomics; a warp per group elects the E most voted workers.  Everything runs in fp64.
+#include "common.cuh"
+#include "locate_common.cuh"
+
+namespace approxifer {
+
+namespace {
+
+using namespace locate_detail;
+
+constexpr int kRowsThreads = 128;
+constexpr int kRowsWarps = kRowsThreads / 32;
+constexpr int kMaxGroupsPerCta = 16;
+
+template <int NMAX, int M>
+struct GroupSmem {
+  static constexpr int MP = (M + 1) / 2 * 2;  // powers padded to pairs: rows stay 16-byte aligned
+  double nt[NMAX - M][NMAX];                  // nt[r][i] = N[i][r]
+  double pw[NMAX][MP];                        // pw[i][k] = b_i^k
+  double xs[NMAX];                            // b_i
+  long long yoff[NMAX];                       // element offset of the i-th available worker's row
+  int votes[NMAX];
+  uint32_t mask;
+  int n;  // workers available; -1: fewer than 2(K+E), nothing to locate
+  uint32_t status;
+  int pad;
+};
+
+template <int NMAX, int M, int K0 = 0>
+__device__ __forceinline__ void rows_pblock_factor(double (&col)[NMAX], int lane, double (*refl)[NMAX]) {
+  if constexpr (K0 < M) {
+    if (lane == K0) make_reflector<NMAX, K0>(col, refl[K0]);
+    __syncwarp();
+    if (lane > K0 && lane < M) apply_reflector<NMAX, K0>(col, refl[K0]);
+    rows_pblock_factor<NMAX, M, K0 + 1>(col, lane, refl);
+  }
+}
+// col <- H_0 H_1 .. H_{M-1} col (reflectors applied last to first)
+template <int NMAX, int M, int K0 = M - 1>
+__device__ __forceinline__ void rows_apply_q(double (&col)[NMAX], double (*refl)[NMAX]) {
+  if constexpr (K0 >= 0) {
+    apply_reflector<NMAX, K0>(col, refl[K0]);
+    rows_apply_q<NMAX, M, K0 - 1>(col, refl);
+  }
+}
+
+// One warp: nodes, powers, reflectors and the complement basis N of one group.
+template <int NMAX, int M>
+__device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double (*refl)[NMAX], const LocateArgs& a,
+                                                 const LocateTables& tab, int64_t g, int lane) {
+  using SM = GroupSmem<NMAX, M>;
+  const uint32_t mask = a.mask[g] & worker_bits(a.W);
+  const int n = __popc(mask);
+  if (lane == 0) {
+    sm.mask = mask;
+    sm.n = (n < 2 * M) ? -1 : n;  // Algorithm 1's condition N-S+1 >= 2(K+E)
+    sm.status = (n < 2 * M) ? kStLocateUnderdetermined : 0u;
+  }
+  if (lane < NMAX) sm.votes[lane] = 0;
+  if (n < 2 * M) return;
+  const int my_worker = (lane < n) ? (int)__fns(mask, 0, lane + 1) : -1;
+  if (lane < NMAX) {
+    const double b = (lane < n) ? tab.beta[my_worker] : 0.0;
+    sm.xs[lane] = b;
+    sm.yoff[lane] = (lane < n) ? (long long)my_worker * a.y_rs : 0;
+    double p = 1.0;
+#pragma unroll
+    for (int k = 0; k < SM::MP; ++k) {
+      sm.pw[lane][k] = (lane < n && k < M) ? p : 0.0;
+      p *= b;
+    }
+  }
+  __syncwarp();
+  double col[NMAX];
+#pragma unroll
+  for (int r = 0; r < NMAX; ++r) col[r] = (lane < M) ? sm.pw[r][lane] : 0.0;
+  rows_pblock_factor<NMAX, M>(col, lane, refl);
+  __syncwarp();
+  // lane r < NMAX-M: column M+r of Q = H_0 .. H_{M-1}
+#pragma unroll
+  for (int r = 0; r < NMAX; ++r) col[r] = (r == M + lane) ? 1.0 : 0.0;
+  if (lane < NMAX - M) {
+    rows_apply_q<NMAX, M>(col, refl);
+#pragma unroll
+    for (int r = 0; r < NMAX; ++r) sm.nt[lane][r] = col[r];
+  }
+}
+
+
+template <int NMAX, int M>
+__global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __grid_constant__ LocateArgs a,
+                                                                      const __grid_constant__ LocateTables tab,
+                                                                      const int gpb) {
+  using SM = GroupSmem<NMAX, M>;
+  constexpr int MP = SM::MP;
+  constexpr int NQ = M - 1;  // unknowns Q_1 .. Q_{M-1}
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  SM* groups = reinterpret_cast<SM*>(smem_raw);
+  // the thread's own predictions, ysm[i][tid]: shared memory rather than registers, which the factor needs
+  // (the same bytes serve, during set-up, as each warp's scratch for the reflectors of the Vandermonde block)
+  unsigned char* scratch = smem_raw + (size_t)gpb * sizeof(SM);
+  float* ysm = reinterpret_cast<float*>(scratch) + threadIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int E = a.E;
+  const int64_t g_first = (int64_t)blockIdx.x * gpb;
+  const int ng = (int)min((int64_t)gpb, a.G - g_first);
+
+  // ---- set-up, one warp per group ------------------------------------------------------------------
+  {
+    double(*refl)[NMAX] = reinterpret_cast<double(*)[NMAX]>(scratch) + warp * M;
+    for (int s = warp; s < ng; s += kRowsWarps) {
+      rows_setup_group<NMAX, M>(groups[s], refl, a, tab, g_first + s, lane);
+      __syncwarp();  // the scratch is reused by this warp's next group
+    }
+  }
+  __syncthreads();
+
+  // ---- one thread per (group, class) -----------------------------------------------------------------
+  const int64_t n_tasks = (int64_t)ng * a.C;
+  for (int64_t t = tid; t < n_tasks; t += kRowsThreads) {
+    const int s = (int)(t / a.C);
+    const int64_t c = t - (int64_t)s * a.C;
+    SM& sm = groups[s];
+    const int n = sm.n;
+    if (n < 0) continue;
+    const float* Yc = a.Yt + (g_first + s) * a.y_gs + c;
+
+#pragma unroll
+    for (int i = 0; i < NMAX; ++i) ysm[i * kRowsThreads] = (i < n) ? __ldg(Yc + sm.yoff[i]) : 0.f;
+
+    // upper-triangular factor R (only j >= k is ever touched) and transformed right-hand side d
+    double R[NQ][NQ], d[NQ];
+#pragma unroll
+    for (int k = 0; k < NQ; ++k) {
+      d[k] = 0.0;
+#pragma unroll
+      for (int j = 0; j < NQ; ++j) R[k][j] = 0.0;
+    }
+
+    const int rows = n - M;
+#pragma unroll 1
+    for (int r = 0; r < rows; ++r) {
+      // row[l] = sum_i N[i][r] y_i b_i^l, l = 0..M-1  (row[0] = b0[r])
+      double row[MP];
+#pragma unroll
+      for (int l = 0; l < MP; ++l) row[l] = 0.0;
+      const double* nr = sm.nt[r];
+#pragma unroll 2
+      for (int i = 0; i < n; i += 2) {  // an odd n reads one padded (zero) entry
+        const double2 nn = *reinterpret_cast<const double2*>(nr + i);
+        const double u0 = nn.x * (double)ysm[i * kRowsThreads], u1 = nn.y * (double)ysm[(i + 1) * kRowsThreads];
+#pragma unroll
+        for (int l = 0; l < MP; l += 2) {
+          const double2 p0 = *reinterpret_cast<const double2*>(&sm.pw[i][l]);
+          const double2 p1 = *reinterpret_cast<const double2*>(&sm.pw[i + 1][l]);
+          row[l] = fma(u0, p0.x, row[l]);
+          row[l + 1] = fma(u0, p0.y, row[l + 1]);
+          row[l] = fma(u1, p1.x, row[l]);
+          row[l + 1] = fma(u1, p1.y, row[l + 1]);
+        }
+      }
+      // fold the equation  sum_k row[k+1] q_k = -row[0]  into (R, d) with Givens rotations
+      double rhs = -row[0];
+#pragma unroll
+      for (int k = 0; k < NQ; ++k) {
+        const double av = R[k][k], bv = row[k + 1];
+        const double h2 = fma(av, av, bv * bv);
+        if (h2 > 0.0) {
+          const double rinv = rsqrt(h2);
+          const double cs = av * rinv, sn = bv * rinv;
+          R[k][k] = h2 * rinv;
+#pragma unroll
+          for (int j = k + 1; j < NQ; ++j) {
+            const double rj = R[k][j], xj = row[j + 1];
+            R[k][j] = fma(cs, rj, sn * xj);
+            row[j + 1] = fma(cs, xj, -sn * rj);
+          }
+          const double dk = d[k];
+          d[k] = fma(cs, dk, sn * rhs);
+          rhs = fma(cs, rhs, -sn * dk);
+        }
+      }
+    }
+
+    // back substitution; an exactly zero pivot leaves its unknown at 0
+    double q[NQ];
+#pragma unroll
+    for (int k = NQ - 1; k >= 0; --k) {
+      double v = d[k];
+#pragma unroll
+      for (int j = k + 1; j < NQ; ++j) v = fma(-R[k][j], q[j], v);
+      q[k] = (R[k][k] != 0.0) ? v / R[k][k] : 0.0;
+    }
+
+    // a_i = Q(b_i) = 1 + sum_k q_k b_i^(k+1); the E smallest |a_i| (ties to the lower worker) get a vote
+    double mag[NMAX];
+    bool nonfinite = false;
+#pragma unroll
+    for (int i = 0; i < NMAX; ++i) {
+      const double b = sm.xs[i];
+      double h = q[NQ - 1];
+#pragma unroll
+      for (int k = NQ - 2; k >= 0; --k) h = fma(h, b, q[k]);
+      const double av = fma(h, b, 1.0);
+      const bool fin = isfinite(av);
+      mag[i] = fin ? fabs(av) : INFINITY;
+      nonfinite |= (i < n) && !fin;
+    }
+    if (nonfinite) atomicOr(&sm.status, kStNonfinite);
+    uint32_t taken = 0;
+    for (int e = 0; e < E; ++e) {
+      int best = -1;
+      double bestv = 0.0;
+#pragma unroll
+      for (int i = 0; i < NMAX; ++i) {
+        const bool cand = (i < n) && !((taken >> i) & 1u) && (best < 0 || mag[i] < bestv);
+        if (cand) {
+          best = i;
+          bestv = mag[i];
+        }
+      }
+      taken |= 1u << best;
+      atomicAdd(&sm.votes[best], 1);
+    }
+  }
+  __syncthreads();
+
+  // ---- the E most voted workers of each group, ties to the lower index; lane = rank ----------------
+  for (int s = warp; s < ng; s += kRowsWarps) {
+    const SM& sm = groups[s];
+    const int64_t g = g_first + s;
+    const uint32_t mask = sm.mask;
+    if (sm.n < 0) {
+      for (int e = lane; e < E; e += 32) a.adv[g * E + e] = -1;
+      if (lane == 0) {
+        a.trusted[g] = mask;
+        if (a.status) a.status[g] = sm.status;
+      }
+      continue;
+    }
+    const int n = sm.n;
+    const int my_worker = (lane < n) ? (int)__fns(mask, 0, lane + 1) : 0;
+    int v = (lane < n) ? sm.votes[lane] : -1;
+    int idx = (lane < n) ? lane : 64 + lane;
+    uint32_t picked = 0;
+    for (int e = 0; e < E; ++e) {
+      const int win = warp_argmin((double)(-v), idx);
+      picked |= 1u << win;
+      if (win == lane) {
+        v = -1;
+        idx = 64 + lane;
+      }
+    }
+    const bool elected = (picked >> lane) & 1u;
+    const uint32_t wbits = __reduce_or_sync(kFull, elected ? (1u << my_worker) : 0u);
+    if (elected) a.adv[g * E + __popc(picked & ((1u << lane) - 1u))] = my_worker;
+    if (lane == 0) {
+      a.trusted[g] = mask & ~wbits;
+      if (a.status) a.status[g] = sm.status;
+    }
+  }
+}
+
+template <int NMAX, int M>
+cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream) {
+  // as many groups per CTA as give every thread a class, within the shared-memory budget of two CTAs per SM
+  int64_t gpb = a.C >= kRowsThreads ? 1 : kRowsThreads / a.C;
+  if (gpb > kMaxGroupsPerCta) gpb = kMaxGroupsPerCta;
+  const size_t per_group = sizeof(GroupSmem<NMAX, M>);
+  size_t y_bytes = (size_t)NMAX * kRowsThreads * sizeof(float);  // per-thread predictions ...
+  const size_t refl_bytes = (size_t)kRowsWarps * M * NMAX * sizeof(double);  // ... aliased with the set-up scratch
+  if (refl_bytes > y_bytes) y_bytes = refl_bytes;
+  while (gpb > 1 && gpb * per_group + y_bytes > 74 * 1024) --gpb;
+  if (gpb > a.G) gpb = a.G;
+  const size_t smem = (size_t)gpb * per_group + y_bytes;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(locate_rows_kernel<NMAX, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  const int64_t blocks = (a.G + gpb - 1) / gpb;
+  if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+  locate_rows_kernel<NMAX, M><<<(unsigned)blocks, kRowsThreads, smem, stream>>>(a, tab, (int)gpb);
+  count_launch();
+  return cudaGetLastError();
+}
+
+template <int NMAX, int M = 2>
+cudaError_t dispatch_rows_m(int m, const LocateArgs& a, const LocateTables& tab, cudaStream_t stream) {
+  if constexpr (M > NMAX / 2 || M > kLocateRowsMaxM) {
+    return cudaErrorInvalidValue;
+  } else {
+    if (m == M) return launch_rows_nm<NMAX, M>(a, tab, stream);
+    return dispatch_rows_m<NMAX, M + 1>(m, a, tab, stream);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_locate_rows(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream) {
+  const int m = a.K + a.E;
+  if (a.W <= 8) return dispatch_rows_m<8>(m, a, tab, stream);
+  if (a.W <= 16) return dispatch_rows_m<16>(m, a, tab, stream);
+  if (a.W <= 24) return dispatch_rows_m<24>(m, a, tab, stream);
+  return dispatch_rows_m<32>(m, a, tab, stream);
+}
+
+}  // namespace approxifer
