@@ -218,6 +218,14 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
 int approxifer_debug_decode_config(int stages, int ctas_per_sm, int disable, int cols, int split);
 
 /*
+ * Test hook for the locator: force_warp_kernel != 0 routes every locate through the
+ * warp-per-group kernel, which otherwise serves only K+E > 10 (smaller K+E use the
+ * thread-per-class kernel).  Both follow Algorithm 2 and return the same sets.
+ * Process-wide, not thread-safe.
+ */
+int approxifer_debug_locate_config(int force_warp_kernel);
+
+/*
  * Every wait on an asynchronous copy inside the kernels is bounded.  Returns how
  * many such waits have given up on the current device since the library was
  * loaded (0 in a correct run; the affected groups' outputs are then

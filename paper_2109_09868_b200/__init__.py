@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     approxifer_locate,
     approxifer_params,
     debug_decode_config,
+    debug_locate_config,
     device_wait_timeouts,
     launch_count,
     library_path,

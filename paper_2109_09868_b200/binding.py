@@ -33,6 +33,7 @@ EXPORTS = (
     "approxifer_launch_count",
     "approxifer_debug_decode_config",
     "approxifer_device_wait_timeouts",
+    "approxifer_debug_locate_config",
     "approxifer_encode_host",
     "approxifer_decode_host",
     "approxifer_locate_host",
@@ -90,6 +91,8 @@ def load() -> ctypes.CDLL:
     lib.approxifer_debug_decode_config.argtypes = [c_int, c_int, c_int, c_int, c_int]
     lib.approxifer_debug_decode_config.restype = c_int
     lib.approxifer_device_wait_timeouts.restype = c_int64
+    lib.approxifer_debug_locate_config.argtypes = [c_int]
+    lib.approxifer_debug_locate_config.restype = c_int
     c_size_t = ctypes.c_size_t
     lib.approxifer_encode_host.argtypes = [pp, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, POINTER(c_void_p), c_int]
     lib.approxifer_encode_host.restype = c_int
@@ -122,6 +125,10 @@ def debug_decode_config(stages: int = 0, ctas_per_sm: int = 0, disable: int = 0,
     rc = load().approxifer_debug_decode_config(int(stages), int(ctas_per_sm), int(disable), int(cols), int(split))
     if rc != OK:
         raise ApproxiferError(rc, "approxifer_debug_decode_config")
+
+
+def debug_locate_config(force_warp_kernel: int = 0) -> None:
+    load().approxifer_debug_locate_config(int(force_warp_kernel))
 
 
 def device_wait_timeouts() -> int:

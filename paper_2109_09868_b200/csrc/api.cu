@@ -99,6 +99,11 @@ int approxifer_debug_decode_config(int stages, int ctas_per_sm, int disable, int
   return APPROXIFER_OK;
 }
 
+int approxifer_debug_locate_config(int force_warp_kernel) {
+  locate_config(force_warp_kernel);
+  return APPROXIFER_OK;
+}
+
 int64_t approxifer_device_wait_timeouts(void) {
   unsigned int n = 0;
   if (read_decode_wait_timeouts(&n) != cudaSuccess) return -1;

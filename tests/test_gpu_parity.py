@@ -433,3 +433,20 @@ def test_worker_major_layouts_for_decode_and_locate():
         out = torch.empty((K, G, C), device=dev())               # query-major output
         ap.approxifer_decode(p, view, trusted, out.permute(1, 0, 2))
         check_decode(K, W, Yt, ref["trusted"], out.permute(1, 0, 2))
+
+
+@pytest.mark.parametrize("K,E,S,W,C", [(8, 2, 2, 24, 10), (3, 2, 1, 12, 37), (4, 1, 2, 12, 300), (2, 1, 0, 6, 1), (7, 3, 1, 22, 10)])
+def test_both_locator_kernels_return_the_same_sets(K, E, S, W, C):
+    """K+E <= 10 normally takes the thread-per-class kernel; the warp-per-group kernel must agree with it
+    (and with the oracle) on the same inputs, including groups with too few workers."""
+    G = 150
+    Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=K + 7 * E + C)
+    mask[5] = (1 << (2 * (K + E) - 1)) - 1  # one worker short: nothing to locate
+    ref, adv_rows, _ = compare_locate(K, W, E, Yt, mask)
+    try:
+        ap.debug_locate_config(1)
+        ref2, adv_warp, _ = compare_locate(K, W, E, Yt, mask)
+    finally:
+        ap.debug_locate_config(0)
+    np.testing.assert_array_equal(adv_rows, adv_warp)
+    assert adv_rows[5, 0] == -1
