@@ -21,8 +21,9 @@
  *     must not overlap.  `params` is a HOST pointer, read during the call.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL =
  *     the legacy default stream) and the call returns without synchronising.
- *     The library allocates no memory, keeps no per-call state and may be
- *     called from several host threads on different streams.
+ *     The library allocates no device memory, keeps no per-call state (only an
+ *     immutable host-side cache of the node tables of each (K, W) seen) and
+ *     may be called from several host threads on different streams.
  *   - 16-byte aligned bases with D (or C) and all strides multiples of 4 take
  *     the 128-bit fast path; anything else runs a slower element-wise GPU
  *     path.  There is no CPU fallback.

@@ -195,8 +195,7 @@ __global__ void debug_encode_weights_kernel(int K, int W, const __grid_constant_
 
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
-  DecodeTables tab;
-  build_decode_tables(a.K, a.W, &tab);
+  const DecodeTables& tab = decode_tables(a.K, a.W);
   const bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&
                    a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
   if (decode_staged_eligible(a)) return launch_decode_staged(a, tab, stream);

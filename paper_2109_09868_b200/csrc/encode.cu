@@ -90,8 +90,7 @@ cudaError_t dispatch_k(const EncodeArgs& a, const EncodeTables& tab, cudaStream_
 
 cudaError_t launch_encode(const EncodeArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
-  EncodeTables tab;
-  build_encode_tables(a.K, a.W, &tab);
+  const EncodeTables& tab = encode_tables(a.K, a.W);
   const bool vec = aligned16(a.X) && aligned16(a.Xt) && a.D % 4 == 0 && a.x_gs % 4 == 0 && a.x_rs % 4 == 0 &&
                    a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
   if (vec) return dispatch_k<float4>(a, tab, stream);

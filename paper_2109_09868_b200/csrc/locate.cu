@@ -270,8 +270,7 @@ void locate_config(int force_warp_kernel) { g_force_warp_kernel = force_warp_ker
 
 cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
-  LocateTables tab;
-  build_locate_tables(a.W, &tab);
+  const LocateTables& tab = locate_tables(a.W);
   const int m = a.K + a.E;
   if (m <= kLocateRowsMaxM && !g_force_warp_kernel) return launch_locate_rows(a, tab, stream);
   if (a.W <= 8) return dispatch_m<8>(m, a, tab, stream);

@@ -3,6 +3,9 @@
 
 #include <cmath>
 #include <cstring>
+#include <map>
+#include <memory>
+#include <mutex>
 
 namespace approxifer {
 
@@ -71,6 +74,39 @@ void build_locate_tables(int W, LocateTables* t) {
   std::memset(t, 0, sizeof(*t));
   // beta_i = cos(pi i/(W-1)) = sin(pi (1/2 - i/(W-1)))
   for (int i = 0; i < W; ++i) t->beta[i] = (double)sinpi_ratio((long long)(W - 1) - 2 * i, 2LL * (W - 1));
+}
+
+namespace {
+
+template <typename T, typename Build>
+const T& cached(std::map<int, std::unique_ptr<T>>& cache, std::mutex& mu, int key, Build build) {
+  std::lock_guard<std::mutex> lock(mu);
+  std::unique_ptr<T>& slot = cache[key];
+  if (!slot) {
+    slot.reset(new T);
+    build(slot.get());
+  }
+  return *slot;
+}
+
+}  // namespace
+
+const EncodeTables& encode_tables(int K, int W) {
+  static std::map<int, std::unique_ptr<EncodeTables>> cache;
+  static std::mutex mu;
+  return cached(cache, mu, K * 64 + W, [&](EncodeTables* t) { build_encode_tables(K, W, t); });
+}
+
+const DecodeTables& decode_tables(int K, int W) {
+  static std::map<int, std::unique_ptr<DecodeTables>> cache;
+  static std::mutex mu;
+  return cached(cache, mu, K * 64 + W, [&](DecodeTables* t) { build_decode_tables(K, W, t); });
+}
+
+const LocateTables& locate_tables(int W) {
+  static std::map<int, std::unique_ptr<LocateTables>> cache;
+  static std::mutex mu;
+  return cached(cache, mu, W, [&](LocateTables* t) { build_locate_tables(W, t); });
 }
 
 }  // namespace approxifer

@@ -40,4 +40,11 @@ void build_encode_tables(int K, int W, EncodeTables* t);
 void build_decode_tables(int K, int W, DecodeTables* t);
 void build_locate_tables(int W, LocateTables* t);
 
+// The tables depend on (K, W) only and cost 10-200 us of host time to build, so each is built once per
+// process and (K, W) and then served from an immutable, mutex-protected cache.  The references stay valid
+// for the life of the process.
+const EncodeTables& encode_tables(int K, int W);
+const DecodeTables& decode_tables(int K, int W);
+const LocateTables& locate_tables(int W);
+
 }  // namespace approxifer
