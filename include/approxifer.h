@@ -133,6 +133,22 @@ int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C,
                       void* cuda_stream);
 
 /*
+ * The decoder's two steps in one call (Section 3, "ApproxIFER Decoding", steps 1 and 2): locate the E
+ * Byzantine workers of every group (Algorithm 2), then decode from the workers that are present and were
+ * not located.  Equivalent to approxifer_locate followed by approxifer_decode with `trusted_mask` as the
+ * mask, enqueued back to back on `cuda_stream`.  `trusted_mask` [G] is required (it carries the result of
+ * step 1 to step 2 on the device); `adv` [G][E], `n_used` [G], `locate_status` [G] and `decode_status` [G]
+ * are as in the two entry points (`adv` is required, the other three may be NULL).
+ */
+int approxifer_locate_decode(const approxifer_params* params, int64_t G, int64_t C,
+                             const float* Yt, int64_t yt_gstride, int64_t yt_rstride,
+                             const uint32_t* mask,
+                             int32_t* adv, uint32_t* trusted_mask,
+                             float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                             int32_t* n_used, uint32_t* locate_status, uint32_t* decode_status,
+                             void* cuda_stream);
+
+/*
  * Host-buffer variants of the three operations (same definitions and citations
  * as above).  Payloads, masks and results live in HOST memory, dense
  * ([G][K][D], [G][W][D], [G][W][C], [G][K][C], [G][E], [G]); pinned memory is

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     approxifer_decode_host,
     approxifer_locate_host,
     approxifer_locate,
+    approxifer_locate_decode,
     approxifer_params,
     debug_decode_config,
     debug_locate_config,

@@ -27,6 +27,7 @@ EXPORTS = (
     "approxifer_encode",
     "approxifer_decode",
     "approxifer_locate",
+    "approxifer_locate_decode",
     "approxifer_debug_weights",
     "approxifer_strerror",
     "approxifer_version",
@@ -82,6 +83,9 @@ def load() -> ctypes.CDLL:
     lib.approxifer_locate.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]
     lib.approxifer_locate.restype = c_int
+    lib.approxifer_locate_decode.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
+                                             c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.approxifer_locate_decode.restype = c_int
     lib.approxifer_debug_weights.argtypes = [pp, c_uint32, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.approxifer_debug_weights.restype = c_int
     lib.approxifer_strerror.argtypes = [c_int]
@@ -213,6 +217,29 @@ def approxifer_locate(params: approxifer_params, Yt: torch.Tensor, mask: torch.T
     if rc != OK:
         raise ApproxiferError(rc, "approxifer_locate")
     return adv, trusted_mask
+
+
+def approxifer_locate_decode(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, Yhat: Optional[torch.Tensor] = None,
+                             n_used: Optional[torch.Tensor] = None, locate_status: Optional[torch.Tensor] = None,
+                             decode_status: Optional[torch.Tensor] = None, stream=None):
+    """Locate the E Byzantine workers of every group, then decode from the remaining present workers.
+    Returns (Yhat [G][K][C], adv [G][E], trusted_mask [G])."""
+    G, W, C = Yt.shape
+    E = max(int(params.E), 0)
+    adv = torch.empty((G, E), device=Yt.device, dtype=torch.int32)
+    trusted = torch.empty((G,), device=Yt.device, dtype=torch.int32)
+    if Yhat is None:
+        Yhat = torch.empty((G, params.K, C), device=Yt.device, dtype=torch.float32)
+    yp, yg, yr = _payload(Yt, params.W, "Yt")
+    op, og, orr = _payload(Yhat, params.K, "Yhat")
+    rc = load().approxifer_locate_decode(ctypes.byref(params), G, C, yp, yg, yr, _vec(mask, torch.int32, G, "mask"),
+                                         adv.data_ptr(), trusted.data_ptr(), op, og, orr,
+                                         _vec(n_used, torch.int32, G, "n_used"),
+                                         _vec(locate_status, torch.int32, G, "locate_status"),
+                                         _vec(decode_status, torch.int32, G, "decode_status"), _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_locate_decode")
+    return Yhat, adv, trusted
 
 
 def approxifer_debug_weights(params: approxifer_params, mask: int = 0, which: int = 0, stream=None):

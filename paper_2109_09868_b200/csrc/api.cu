@@ -81,6 +81,22 @@ int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C, con
   return from_cuda(launch_locate(a, static_cast<cudaStream_t>(cuda_stream)));
 }
 
+int approxifer_locate_decode(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
+                             int64_t yt_rstride, const uint32_t* mask, int32_t* adv, uint32_t* trusted_mask, float* Yhat,
+                             int64_t yh_gstride, int64_t yh_rstride, int32_t* n_used, uint32_t* locate_status,
+                             uint32_t* decode_status, void* cuda_stream) {
+  // validate both steps before anything is enqueued
+  if (G > 0 && Yhat == nullptr) return APPROXIFER_E_NULL;
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if ((rc = check_layout(G, C, yh_rstride))) return rc;
+  if (yh_gstride < 0) return APPROXIFER_E_RANGE;
+  rc = approxifer_locate(params, G, C, Yt, yt_gstride, yt_rstride, mask, adv, trusted_mask, locate_status, cuda_stream);
+  if (rc) return rc;
+  return approxifer_decode(params, G, C, Yt, yt_gstride, yt_rstride, trusted_mask, Yhat, yh_gstride, yh_rstride, n_used,
+                           decode_status, cuda_stream);
+}
+
 int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int which, float* w, int32_t* idx,
                              int32_t* n, void* cuda_stream) {
   int rc = check_kw(params);

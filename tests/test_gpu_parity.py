@@ -450,3 +450,22 @@ def test_both_locator_kernels_return_the_same_sets(K, E, S, W, C):
         ap.debug_locate_config(0)
     np.testing.assert_array_equal(adv_rows, adv_warp)
     assert adv_rows[5, 0] == -1
+
+
+def test_locate_decode_in_one_call_equals_the_two_steps():
+    K, E, S, W, G, C = 8, 2, 2, 24, 300, 10
+    Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=21)
+    mask[7] = 0x3FF  # too few workers: nothing located, decoded from all ten
+    p = ap.make_params(K, W, E)
+    Yd, md = Yt.to(dev()), ap.mask_tensor(mask)
+    n_used = torch.empty(G, dtype=torch.int32, device=dev())
+    lst = torch.empty(G, dtype=torch.int32, device=dev())
+    dst = torch.empty(G, dtype=torch.int32, device=dev())
+    Yh, adv, trusted = ap.approxifer_locate_decode(p, Yd, md, n_used=n_used, locate_status=lst, decode_status=dst)
+    adv2, trusted2 = ap.approxifer_locate(p, Yd, md)
+    Yh2 = ap.approxifer_decode(p, Yd, trusted2)
+    assert torch.equal(adv, adv2) and torch.equal(trusted, trusted2) and torch.equal(Yh, Yh2)
+    ref = oracle.locate(K, W, E, Yt.numpy(), mask)
+    np.testing.assert_array_equal(adv.cpu().numpy(), ref["adv"])
+    check_decode(K, W, Yt, ref["trusted"], Yh, n_used, dst)
+    assert int(lst[7]) == 4 and int(n_used[7]) == 10
