@@ -479,3 +479,15 @@ def test_locate_then_decode_recovers_linear_predictions():
     assert np.abs(Yh - clean).max() < 0.5
     Yh_bad, _, _ = oracle.decode(K, W, Y, mask)
     assert np.abs(Yh_bad - clean).max() > 2.0
+
+
+def test_locate_exact_ties_in_magnitude_go_to_the_lower_worker():
+    """A class whose predictions are all zero leaves Q = 1, so every a_i equals 1 exactly: the tie rule
+    alone decides, and it must pick the E lowest present workers (Algorithm 2 is silent; ties -> lower index)."""
+    K, E, W, C = 3, 2, 12, 3
+    Y = np.zeros((2, W, C), dtype=np.float32)
+    mask = np.array([0xFFF, 0xFFC | 0x0], dtype=np.uint32)  # second group: workers 0 and 1 absent
+    out = oracle.locate(K, W, E, Y, mask)
+    assert list(out["adv"][0]) == [0, 1]
+    assert list(out["adv"][1]) == [2, 3]
+    assert out["min_gap"][0] == 1.0 and out["vote_margin"][0] == C
