@@ -200,6 +200,15 @@ def run_reference(args):
 
 # ---------------------------------------------------------------- GPU measuring
 
+def physical_gpu_index(local_rank: int) -> int:
+    """nvidia-smi index of this rank's GPU (CUDA_VISIBLE_DEVICES may renumber the devices)."""
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    ids = [v.strip() for v in vis.split(",") if v.strip()]
+    if local_rank < len(ids) and ids[local_rank].isdigit():
+        return int(ids[local_rank])
+    return local_rank
+
+
 def time_launches(fn, warmup=3, iters=10):
     """Per-launch device time (ms) of fn() on the current stream: median and min."""
     for _ in range(warmup):
@@ -464,8 +473,7 @@ def main():
         step()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
-                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]) if os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank].isdigit() else local_rank)
+    sampler = ClockSampler(physical_gpu_index(local_rank))
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -490,6 +498,26 @@ def main():
     dec_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
     ms_per_step = total_ms / args.steps
     value = world * (enc_b + dec_b) / ms_per_step / 1e6
+
+    # end to end through the host-buffer entry points, on every rank (max over ranks, like the device figure)
+    e2e = None
+    if not args.no_e2e and args.groups is None:
+        del X, Xt
+        torch.cuda.empty_cache()
+        try:
+            ms, h2d, d2h, l_e2e = run_e2e(ap, dev, w, mask_np, steps=3, warmup=1)
+        except RuntimeError as exc:  # e.g. not enough pinned host memory for every rank
+            ms, h2d, d2h, l_e2e = float("inf"), 0, 0, 0
+            sys.stderr.write("rank %d: end-to-end measurement failed: %s\n" % (rank, exc))
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        if ms != float("inf"):
+            e2e = {"value": world * (enc_b + dec_b) / ms / 1e6, "unit": UNIT, "ms_per_step": ms,
+                   "h2d_bytes_per_step": world * h2d, "d2h_bytes_per_step": world * d2h, "gpu_launches_per_step": world * l_e2e,
+                   "note": "approxifer_encode_host + approxifer_decode_host on every rank, pinned host buffers, 512 MiB device "
+                           "workspace, 4 streams; PCIe-bound"}
 
     if rank != 0:
         if world > 1:
@@ -518,19 +546,9 @@ def main():
     }
     if cpu is not None:
         line["cpu_baseline"] = cpu
-    if not args.no_e2e and world == 1 and args.groups is None:
-        del X, Xt
-        torch.cuda.empty_cache()
-        ms, h2d, d2h, l_e2e = run_e2e(ap, dev, w, mask_np, steps=3, warmup=1)
-        line["e2e"] = {"value": (enc_b + dec_b) / ms / 1e6, "unit": UNIT, "ms_per_step": ms, "h2d_bytes_per_step": h2d,
-                       "d2h_bytes_per_step": d2h, "gpu_launches_per_step": l_e2e,
-                       "note": "approxifer_encode_host + approxifer_decode_host, pinned host buffers, 512 MiB device workspace, 4 streams; PCIe-bound"}
-    elif world > 1 or args.no_e2e or args.groups is not None:
-        line["e2e"] = None
+    line["e2e"] = e2e
     if not args.no_others and world == 1 and args.groups is None:
-        for name in ("X", "Xt", "Yt", "Yh"):
-            if name in locals():
-                del locals()[name]
+        del Yt, Yh
         torch.cuda.empty_cache()
         line["others"] = other_workloads(ap, dev, peak)
     print(json.dumps(line), flush=True)
