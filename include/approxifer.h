@@ -13,7 +13,8 @@
  * query / per prediction.  Nodes (Section 3, "Encoding"):
  *     alpha_j = cos((2j+1) pi / (2K)),      beta_i = cos(i pi / (W-1)).
  *
- * Common rules for every entry point
+ * Common rules for every entry point (the *_host variants further down take
+ * HOST arrays instead and say so)
  *   - All array arguments are DEVICE pointers owned by the caller (global
  *     memory of the current device), fp32 payloads, innermost dimension
  *     contiguous; "gstride" / "rstride" are the distances, in ELEMENTS, between
@@ -21,9 +22,11 @@
  *     must not overlap.  `params` is a HOST pointer, read during the call.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL =
  *     the legacy default stream) and the call returns without synchronising.
- *     The library allocates no device memory, keeps no per-call state (only an
- *     immutable host-side cache of the node tables of each (K, W) seen) and
- *     may be called from several host threads on different streams.
+ *     The library never allocates device memory (its image contains one fixed
+ *     staging array, see approxifer_encode_host_static), keeps no per-call
+ *     state (only an immutable host-side cache of the node tables of each
+ *     (K, W) seen) and may be called from several host threads on different
+ *     streams.
  *   - 16-byte aligned bases with D (or C) and all strides multiples of 4 take
  *     the 128-bit fast path; anything else runs a slower element-wise GPU
  *     path.  There is no CPU fallback.
