@@ -41,8 +41,12 @@ template <int K, typename V>
 __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_constant__ DecodeArgs a,
                                                                 const __grid_constant__ DecodeTables tab) {
   using Ops = Vec<V>;
-  __shared__ float s_rg[kMaxW * K];  // [i][j] = 1/(alpha_j - beta_i)
-  for (int idx = threadIdx.x; idx < a.W * K; idx += kDecodeThreads) s_rg[idx] = tab.rg[idx];
+  constexpr int KP = (K + 3) / 4 * 4;              // table rows padded to whole float4s
+  __shared__ __align__(16) float s_rg[kMaxW * KP];  // [i][j] = 1/(alpha_j - beta_i), 0 beyond K
+  for (int idx = threadIdx.x; idx < a.W * KP; idx += kDecodeThreads) {
+    const int i = idx / KP, j = idx - i * KP;
+    s_rg[idx] = (j < K) ? tab.rg[i * K + j] : 0.f;
+  }
   __syncthreads();
 
   const uint32_t Cv = (uint32_t)(a.C / Ops::kLanes);
@@ -73,7 +77,12 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
   auto use_row = [&](int i, int r, V y) {
     const float sgn = ((literal ? i : r) & 1) ? -1.f : 1.f;
     const V ys = Ops::scale(sgn, y);
-    const float* rg = s_rg + i * K;
+    float rg[KP];
+#pragma unroll
+    for (int q = 0; q < KP / 4; ++q) {
+      const float4 w4 = *reinterpret_cast<const float4*>(s_rg + i * KP + 4 * q);
+      rg[4 * q] = w4.x, rg[4 * q + 1] = w4.y, rg[4 * q + 2] = w4.z, rg[4 * q + 3] = w4.w;
+    }
     if (!any_coin) {
 #pragma unroll
       for (int j = 0; j < K; ++j) {
@@ -94,24 +103,45 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
     }
   };
 
-  // Walk the present workers in ascending order, four rows in flight at a time.
-  uint32_t m = mask;
-  int r = 0;
-  while (m) {
-    int i[4];
-    V y[4];
+  // Walk the present workers in ascending order.
+  if (Ops::kLanes == 1) {
+    // 4-byte columns (narrow or unaligned payloads): sweep the W workers eight at a time; the loads of the
+    // present ones are issued together, then consumed in ascending order (r counts the present workers).
+    int r = 0;
+    for (int i0 = 0; i0 < a.W; i0 += 8) {
+      const uint32_t bits = (mask >> i0) & 0xffu;
+      if (bits == 0) continue;
+      V y[8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      i[u] = m ? (__ffs(m) - 1) : -1;
-      m &= m - 1;  // 0 stays 0
+      for (int u = 0; u < 8; ++u)
+        if ((bits >> u) & 1u) y[u] = ld_stream(in + (i0 + u) * in_rs);
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if ((bits >> u) & 1u) {
+          use_row(i0 + u, r, y[u]);
+          ++r;
+        }
     }
+  } else {
+    // 16-byte columns: four rows in flight at a time.
+    uint32_t m = mask;
+    int r = 0;
+    while (m) {
+      int i[4];
+      V y[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (i[u] >= 0) y[u] = ld_stream(in + i[u] * in_rs);
+      for (int u = 0; u < 4; ++u) {
+        i[u] = m ? (__ffs(m) - 1) : -1;
+        m &= m - 1;  // 0 stays 0
+      }
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (i[u] >= 0) use_row(i[u], r + u, y[u]);
-    r += 4;
+      for (int u = 0; u < 4; ++u)
+        if (i[u] >= 0) y[u] = ld_stream(in + i[u] * in_rs);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (i[u] >= 0) use_row(i[u], r + u, y[u]);
+      r += 4;
+    }
   }
 
   V* out = reinterpret_cast<V*>(a.Yh + g * a.o_gs) + v;
@@ -124,7 +154,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
     else if ((pinned >> j) & 1u)
       o = acc[j];
     else
-      o = Ops::scale(1.0f / den[j], acc[j]);
+      o = Ops::scale(__frcp_rn(den[j]), acc[j]);  // correctly rounded, like 1.0f / den
     st_stream(out + j * out_rs, o);
   }
   if (v == 0) {
