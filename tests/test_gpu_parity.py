@@ -469,3 +469,72 @@ def test_locate_decode_in_one_call_equals_the_two_steps():
     np.testing.assert_array_equal(adv.cpu().numpy(), ref["adv"])
     check_decode(K, W, Yt, ref["trusted"], Yh, n_used, dst)
     assert int(lst[7]) == 4 and int(n_used[7]) == 10
+
+
+# ------------------------------------------------------------------ randomized shapes
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_strides_and_alignments(seed):
+    """Seeded random (K, W, G, length, padding, base offset): every kernel path (128-bit, element-wise, staged)
+    against the oracle, with canaries around and between the rows."""
+    rng = np.random.default_rng(1000 + seed)
+    K = int(rng.integers(1, 33))
+    W = int(rng.integers(2, 33))
+    G = int(rng.integers(1, 40))
+    L = int(rng.choice([1, 2, 3, 5, 8, 12, 31, 64, 100, 257, 512, 516, 640, 1000, 1028, 2052]))
+    pad = int(rng.choice([0, 0, 4, 8, 1, 3]))
+    off = int(rng.choice([0, 0, 4, 1]))
+    g = torch.Generator().manual_seed(seed)
+
+    def guarded(rows):
+        buf = torch.full((off + G * rows * (L + pad) + 7,), CANARY, device=dev())
+        view = buf[off: off + G * rows * (L + pad)].view(G, rows, L + pad)[:, :, :L]
+        return buf, view
+
+    # encode
+    X = torch.rand((G, K, L), generator=g) * 2 - 1
+    xin_buf, xin = guarded(K)
+    xin.copy_(X.to(dev()))
+    out_buf, out = guarded(W)
+    ap.approxifer_encode(ap.make_params(K, W), xin, out)
+    check_encode(K, W, X, out)
+    chk = out_buf.clone()
+    chk[off: off + G * W * (L + pad)].view(G, W, L + pad)[:, :, :L] = CANARY
+    assert bool((chk == CANARY).all())
+    # decode
+    Yt = torch.randn((G, W, L), generator=g)
+    mask = random_masks(W, G, rng, min_present=0)
+    yin_buf, yin = guarded(W)
+    yin.copy_(Yt.to(dev()))
+    for gi in range(G):  # absent rows hold NaN
+        for i in range(W):
+            if not (int(mask[gi]) >> i) & 1:
+                yin[gi, i] = float("nan")
+    yh_buf, yh = guarded(K)
+    n_used = torch.empty(G, dtype=torch.int32, device=dev())
+    status = torch.empty(G, dtype=torch.int32, device=dev())
+    ap.approxifer_decode(ap.make_params(K, W), yin, ap.mask_tensor(mask), yh, n_used=n_used, status=status)
+    check_decode(K, W, Yt, mask, yh, n_used, status)
+    chk = yh_buf.clone()
+    chk[off: off + G * K * (L + pad)].view(G, K, L + pad)[:, :, :L] = CANARY
+    assert bool((chk == CANARY).all())
+    assert ap.device_wait_timeouts() == 0
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_locator_shapes(seed):
+    """Seeded random (K, E, S, C) through both locator kernels' ranges; the located set equals the oracle's on
+    every group that is not near-tied, and whatever is returned is a valid answer."""
+    rng = np.random.default_rng(500 + seed)
+    while True:
+        K = int(rng.integers(1, 14))
+        E = int(rng.integers(1, 4))
+        S = int(rng.integers(0, 4))
+        W = 2 * (K + E) + S
+        if W <= 32:
+            break
+    C = int(rng.choice([1, 2, 7, 10, 33, 130]))
+    G = int(rng.integers(5, 60))
+    Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=seed, softmax=bool(seed % 3 == 0))
+    mask[0] = 2**W - 1  # all workers present in one group
+    compare_locate(K, W, E, Yt, mask, allow_fragile=True)
