@@ -175,6 +175,8 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
     int32_t tile_batch = tile;
     uint32_t mask_batch = 0;
     int64_t k = 0;
+    int stage = 0;
+    uint32_t phase = 1;  // parity of the slot's previous "empty" phase; first used on the second lap of the ring
     for (; k < my_items; ++k) {
       if ((k & 31) == 0) {
         // lane l fetches the mask of item k + l: its group is g_batch advanced l times
@@ -187,12 +189,11 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
         g_batch += dq * 32 + t32 / plan.tiles;
         tile_batch = (int32_t)(t32 % plan.tiles);
       }
-      const int stage = (int)(k % S);
-      if (k >= S && !wait(empty + stage, (uint32_t)(((k / S) - 1) & 1))) break;  // compute warps are done with the slot
+      if (k >= S && !wait(empty + stage, phase)) break;  // compute warps are done with the slot
       const uint32_t col0 = (uint32_t)tile * COLS;
       const uint32_t row_bytes = min((uint32_t)COLS, Cv - col0) * 16u;
       unsigned char* mb = slots + (size_t)stage * slot_sz;
-      int32_t* hdr = reinterpret_cast<int32_t*>(mb);  // [0] = n
+      int32_t* hdr = reinterpret_cast<int32_t*>(mb);  // [0] = n, [1] = first column, [2..3] = group
       float* inv_den = reinterpret_cast<float*>(mb + 16);
       float* w = reinterpret_cast<float*>(mb + kWeightsOff);
       const uint32_t m = __shfl_sync(kFull, mask_batch, (int)(k & 31)) & wb;
@@ -224,6 +225,8 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
       }
       if (lane == 0) {
         hdr[0] = n;
+        hdr[1] = (int32_t)col0;
+        *reinterpret_cast<int64_t*>(hdr + 2) = g;
         if (col0 == 0) {
           if (a.n_used) a.n_used[g] = n;
           if (a.status) a.status[g] = (n == 0 ? kStNoWorkers : 0u) | (n < K ? kStFewWorkers : 0u);
@@ -248,6 +251,10 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
       __syncwarp();  // the whole item block is written before lane 0 publishes it
       if (lane == 0) mbar_arrive(bar);
       // next item of this CTA
+      if (++stage == S) {
+        stage = 0;
+        phase ^= 1u;
+      }
       g += dq;
       tile += dr;
       if (tile >= plan.tiles) {
@@ -266,18 +273,20 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
   const int half = tid / COLS;
   const uint32_t col = (uint32_t)(tid - half * COLS);
 
+  int stage = 0;
+  uint32_t phase = 0;
   for (int64_t k = 0; k < my_items; ++k) {
-    const int stage = (int)(k % S);
-    if (!wait(full + stage, (uint32_t)((k / S) & 1))) {
+    if (!wait(full + stage, phase)) {
       give_up();
       return;
     }
-    const int64_t item = first + k * stride;
-    const int64_t g = item / plan.tiles;
-    const uint32_t col0 = (uint32_t)(item - g * plan.tiles) * COLS;
-    const uint32_t ncols = min((uint32_t)COLS, Cv - col0);
+    // the producer left the item's coordinates in the slot's header
     const unsigned char* mb = slots + (size_t)stage * slot_sz;
-    const int n = *reinterpret_cast<const int32_t*>(mb);
+    const int4 hdr = *reinterpret_cast<const int4*>(mb);
+    const int n = hdr.x;
+    const uint32_t col0 = (uint32_t)hdr.y;
+    const int64_t g = (int64_t)(((uint64_t)(uint32_t)hdr.w << 32) | (uint32_t)hdr.z);
+    const uint32_t ncols = min((uint32_t)COLS, Cv - col0);
     const float* inv_den = reinterpret_cast<const float*>(mb + 16);
     // idle threads (beyond the last column) shadow column 0 and store nothing
     const bool active = col < ncols;
@@ -327,6 +336,10 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
     // this warp no longer needs the slot
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(empty + stage));
+    if (++stage == S) {
+      stage = 0;
+      phase ^= 1u;
+    }
 
     float4* out = reinterpret_cast<float4*>(a.Yh + g * a.o_gs) + col0 + col;
     const int64_t out_rs = a.o_rs / 4;
