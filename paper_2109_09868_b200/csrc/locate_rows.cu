@@ -58,10 +58,116 @@ __device__ __forceinline__ void rows_apply_q(double (&col)[NMAX], double (*refl)
   }
 }
 
-// One warp: nodes, powers, reflectors and the complement basis N of one group.
+// Index of the r-th (0-based) set bit of m; r < popc(m).  Five halving steps on population counts.
+__device__ __forceinline__ int nth_set_bit(uint32_t m, int r) {
+  int pos = 0;
+#pragma unroll
+  for (int w = 16; w > 0; w >>= 1) {
+    const uint32_t low = m & ((1u << w) - 1u);
+    const int c = __popc(low);
+    const bool up = r >= c;
+    r = up ? r - c : r;
+    m = up ? (m >> w) : low;
+    pos += up ? w : 0;
+  }
+  return pos;
+}
+
+// 1/sqrt(h) for a positive, normal h: hardware seed (about 23 bits) and two Newton steps, no special cases.
+// The Givens rotations only need cs^2 + sn^2 = 1 to rounding, which this gives.
+__device__ __forceinline__ double rsqrt_pos(double h) {
+  double y;
+  asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(h));
+  const double hh = 0.5 * h;
+  double e = fma(-hh * y, y, 0.5);
+  y = fma(y, e, y);
+  e = fma(-hh * y, y, 0.5);
+  y = fma(y, e, y);
+  return y;
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+  return v;  // the same value, bit for bit, in every lane
+}
+
+// The complement basis of a group with only a few workers missing, derived from the basis Nf of the full node
+// set.  A vector that is orthogonal to the polynomials on the available nodes is, padded with zeros at the
+// missing nodes, orthogonal to them on all nodes; so the group's complement is { Nf c : (Nf c)_i = 0 for every
+// missing i }, and with Q = H_0 .. H_{s-1} the Householder factor of the (W-M) x s matrix of the missing
+// workers' rows of Nf, the columns s .. W-M-1 of Nf Q restricted to the available workers are an orthonormal
+// basis of it.  Cost: s small reflectors of length W-M (lane = column of Nf) and their application to one row of
+// Nf per lane (lane = available worker), instead of M reflectors of length n and n-M long back-transformations.
+//   nft[d * NMAX + i] = Nf[i][d] (zero beyond W or W-M), vq: scratch of SMAX * (NMAX-M) doubles.
 template <int NMAX, int M>
-__device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double (*refl)[NMAX], const LocateArgs& a,
-                                                 const LocateTables& tab, int64_t g, int lane) {
+__device__ __forceinline__ void rows_basis_from_full(GroupSmem<NMAX, M>& sm, const double* nft, double* vq, uint32_t mask,
+                                                     int W, int n, int my_worker, int lane) {
+  constexpr int DN = NMAX - M;
+  constexpr int SMAX = M / 2 + 1;
+  const int s = W - n;
+  const uint32_t absent = ~mask & worker_bits(W);
+  if (s > 0) {
+    double arow[SMAX];  // lane = d: arow[t] = Nf[t-th missing worker][d]
+#pragma unroll
+    for (int t = 0; t < SMAX; ++t) {
+      const int it = (t < s) ? nth_set_bit(absent, t) : 0;
+      arow[t] = (t < s && lane < DN) ? nft[lane * NMAX + it] : 0.0;
+    }
+#pragma unroll
+    for (int t = 0; t < SMAX; ++t) {
+      if (t < s) {  // uniform over the warp
+        const double x = (lane >= t) ? arow[t] : 0.0;
+        const double s2 = warp_sum(x * x);
+        const double x0 = __shfl_sync(kFull, arow[t], t);
+        const bool nz = s2 > 0.0;
+        const double normx = nz ? s2 * rsqrt(s2) : 0.0;
+        const double akk = (x0 >= 0.0) ? -normx : normx;
+        const double c = fma(fabs(x0), normx, s2);
+        const double scale = nz ? rsqrt(c) : 0.0;
+        const double v = (lane == t) ? (x0 - akk) * scale : x * scale;
+        if (lane < DN) vq[t * DN + lane] = v;
+#pragma unroll
+        for (int t2 = t + 1; t2 < SMAX; ++t2) {
+          if (t2 < s) {
+            const double dot = warp_sum(v * arow[t2]);
+            arow[t2] = fma(-dot, v, arow[t2]);
+          }
+        }
+      }
+    }
+    __syncwarp();
+  }
+  // lane = rank of an available worker: its row of Nf, times H_0 .. H_{s-1}
+  if (lane < NMAX) {
+    double x[DN];
+#pragma unroll
+    for (int d = 0; d < DN; ++d) x[d] = (lane < n) ? nft[d * NMAX + my_worker] : 0.0;
+#pragma unroll
+    for (int t = 0; t < SMAX; ++t) {
+      if (t < s) {
+        const double* v = vq + t * DN;
+        double da = 0.0, db = 0.0;
+#pragma unroll
+        for (int d = 0; d < DN; d += 2) {
+          da = fma(x[d], v[d], da);
+          if (d + 1 < DN) db = fma(x[d + 1], v[d + 1], db);
+        }
+        const double dot = -(da + db);
+#pragma unroll
+        for (int d = 0; d < DN; ++d) x[d] = fma(dot, v[d], x[d]);
+      }
+    }
+#pragma unroll
+    for (int d = 0; d < DN; ++d)
+      if (d >= s) sm.nt[d - s][lane] = x[d];
+  }
+}
+
+// One warp: nodes, powers and the complement basis N of one group.
+template <int NMAX, int M>
+__device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double (*refl)[NMAX], const double* nft,
+                                                 const LocateArgs& a, const LocateTables& tab, int64_t g, int lane) {
   using SM = GroupSmem<NMAX, M>;
   const uint32_t mask = a.mask[g] & worker_bits(a.W);
   const int n = __popc(mask);
@@ -72,7 +178,7 @@ __device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double 
   }
   if (lane < NMAX) sm.votes[lane] = 0;
   if (n < 2 * M) return;
-  const int my_worker = (lane < n) ? (int)__fns(mask, 0, lane + 1) : -1;
+  const int my_worker = (lane < n) ? nth_set_bit(mask, lane) : -1;
   if (lane < NMAX) {
     const double b = (lane < n) ? tab.beta[my_worker] : 0.0;
     sm.xs[lane] = b;
@@ -85,6 +191,11 @@ __device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double 
     }
   }
   __syncwarp();
+  if (a.W - n <= M / 2 + 1) {
+    rows_basis_from_full<NMAX, M>(sm, nft, &refl[0][0], mask, a.W, n, my_worker, lane);
+    return;
+  }
+  // many workers missing: Householder reflectors of the group's own Vandermonde block, applied to unit vectors
   double col[NMAX];
 #pragma unroll
   for (int r = 0; r < NMAX; ++r) col[r] = (lane < M) ? sm.pw[r][lane] : 0.0;
@@ -104,6 +215,7 @@ __device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double 
 template <int NMAX, int M>
 __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __grid_constant__ LocateArgs a,
                                                                       const __grid_constant__ LocateTables tab,
+                                                                      const __grid_constant__ LocateBasis basis,
                                                                       const int gpb) {
   using SM = GroupSmem<NMAX, M>;
   constexpr int MP = SM::MP;
@@ -121,9 +233,17 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
 
   // ---- set-up, one warp per group ------------------------------------------------------------------
   {
+    // the full-set basis, transposed and zero-padded, behind the warps' reflector scratch
+    double* nft = reinterpret_cast<double*>(scratch) + kRowsWarps * M * NMAX;
+    const int dn = a.W - M;
+    for (int idx = tid; idx < (NMAX - M) * NMAX; idx += kRowsThreads) {
+      const int d = idx / NMAX, i = idx - d * NMAX;
+      nft[idx] = (d < dn && i < a.W) ? basis.nfull[i * dn + d] : 0.0;
+    }
+    __syncthreads();
     double(*refl)[NMAX] = reinterpret_cast<double(*)[NMAX]>(scratch) + warp * M;
     for (int s = warp; s < ng; s += kRowsWarps) {
-      rows_setup_group<NMAX, M>(groups[s], refl, a, tab, g_first + s, lane);
+      rows_setup_group<NMAX, M>(groups[s], refl, nft, a, tab, g_first + s, lane);
       __syncwarp();  // the scratch is reused by this warp's next group
     }
   }
@@ -179,8 +299,8 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
       for (int k = 0; k < NQ; ++k) {
         const double av = R[k][k], bv = row[k + 1];
         const double h2 = fma(av, av, bv * bv);
-        if (h2 > 0.0) {
-          const double rinv = rsqrt(h2);
+        if (h2 > 1e-290) {  // (an exactly zero column leaves the factor as it is)
+          const double rinv = rsqrt_pos(h2);
           const double cs = av * rinv, sn = bv * rinv;
           R[k][k] = h2 * rinv;
 #pragma unroll
@@ -253,7 +373,7 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
       continue;
     }
     const int n = sm.n;
-    const int my_worker = (lane < n) ? (int)__fns(mask, 0, lane + 1) : 0;
+    const int my_worker = (lane < n) ? nth_set_bit(mask, lane) : 0;
     int v = (lane < n) ? sm.votes[lane] : -1;
     int idx = (lane < n) ? lane : 64 + lane;
     uint32_t picked = 0;
@@ -282,7 +402,8 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
   if (gpb > kMaxGroupsPerCta) gpb = kMaxGroupsPerCta;
   const size_t per_group = sizeof(GroupSmem<NMAX, M>);
   size_t y_bytes = (size_t)NMAX * kRowsThreads * sizeof(float);  // per-thread predictions ...
-  const size_t refl_bytes = (size_t)kRowsWarps * M * NMAX * sizeof(double);  // ... aliased with the set-up scratch
+  // ... aliased with the set-up scratch: the warps' reflectors and the transposed full-set basis
+  const size_t refl_bytes = ((size_t)kRowsWarps * M + (NMAX - M)) * NMAX * sizeof(double);
   if (refl_bytes > y_bytes) y_bytes = refl_bytes;
   while (gpb > 1 && gpb * per_group + y_bytes > 74 * 1024) --gpb;
   if (gpb > a.G) gpb = a.G;
@@ -293,7 +414,7 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
   }
   const int64_t blocks = (a.G + gpb - 1) / gpb;
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-  locate_rows_kernel<NMAX, M><<<(unsigned)blocks, kRowsThreads, smem, stream>>>(a, tab, (int)gpb);
+  locate_rows_kernel<NMAX, M><<<(unsigned)blocks, kRowsThreads, smem, stream>>>(a, tab, locate_basis(a.W, M), (int)gpb);
   count_launch();
   return cudaGetLastError();
 }

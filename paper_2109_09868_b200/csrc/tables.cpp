@@ -76,6 +76,48 @@ void build_locate_tables(int W, LocateTables* t) {
   for (int i = 0; i < W; ++i) t->beta[i] = (double)sinpi_ratio((long long)(W - 1) - 2 * i, 2LL * (W - 1));
 }
 
+void build_locate_basis(int W, int M, LocateBasis* t) {
+  std::memset(t, 0, sizeof(*t));
+  t->cols = W - M;
+  if (M < 1 || M >= W) return;
+  // Householder QR of the W x M matrix [T_k(beta_i)] (Chebyshev polynomials: the same column spaces as the
+  // monomials, far better conditioned), in extended precision.  Columns M .. W-1 of Q = H_0 .. H_{M-1} are
+  // the basis.
+  long double a[kMaxW][kMaxW];  // a[i][k]
+  long double v[kMaxW][kMaxW];  // v[k][i]: reflector k, H_k = I - v v^T with |v|^2 = 2
+  for (int i = 0; i < W; ++i) {
+    const long double b = sinpi_ratio((long long)(W - 1) - 2 * i, 2LL * (W - 1));
+    a[i][0] = 1.0L;
+    if (M > 1) a[i][1] = b;
+    for (int k = 2; k < M; ++k) a[i][k] = 2.0L * b * a[i][k - 1] - a[i][k - 2];
+  }
+  for (int k = 0; k < M; ++k) {
+    long double s2 = 0.0L;
+    for (int i = k; i < W; ++i) s2 += a[i][k] * a[i][k];
+    const long double normx = sqrtl(s2);
+    const long double x0 = a[k][k];
+    const long double akk = (x0 >= 0.0L) ? -normx : normx;
+    const long double c = s2 + fabsl(x0) * normx;
+    const long double scale = (c > 0.0L) ? 1.0L / sqrtl(c) : 0.0L;
+    for (int i = 0; i < W; ++i) v[k][i] = (i < k) ? 0.0L : ((i == k) ? (x0 - akk) * scale : a[i][k] * scale);
+    for (int j = k; j < M; ++j) {
+      long double dot = 0.0L;
+      for (int i = k; i < W; ++i) dot += v[k][i] * a[i][j];
+      for (int i = k; i < W; ++i) a[i][j] -= dot * v[k][i];
+    }
+  }
+  for (int d = 0; d < W - M; ++d) {
+    long double q[kMaxW];
+    for (int i = 0; i < W; ++i) q[i] = (i == M + d) ? 1.0L : 0.0L;
+    for (int k = M - 1; k >= 0; --k) {
+      long double dot = 0.0L;
+      for (int i = k; i < W; ++i) dot += v[k][i] * q[i];
+      for (int i = k; i < W; ++i) q[i] -= dot * v[k][i];
+    }
+    for (int i = 0; i < W; ++i) t->nfull[i * (W - M) + d] = (double)q[i];
+  }
+}
+
 namespace {
 
 template <typename T, typename Build>
@@ -107,6 +149,12 @@ const LocateTables& locate_tables(int W) {
   static std::map<int, std::unique_ptr<LocateTables>> cache;
   static std::mutex mu;
   return cached(cache, mu, W, [&](LocateTables* t) { build_locate_tables(W, t); });
+}
+
+const LocateBasis& locate_basis(int W, int M) {
+  static std::map<int, std::unique_ptr<LocateBasis>> cache;
+  static std::mutex mu;
+  return cached(cache, mu, W * 64 + M, [&](LocateBasis* t) { build_locate_basis(W, M, t); });
 }
 
 }  // namespace approxifer

@@ -29,6 +29,14 @@ struct LocateTables {
   double beta[kMaxW];
 };
 
+// Orthonormal basis of the orthogonal complement of {polynomials of degree < M} on the FULL node set
+// beta_0 .. beta_{W-1} (all workers present): nfull[i * cols + d], cols = W - M.  The locator derives the
+// basis of a group with a few workers missing from this one instead of factorising from scratch.
+struct LocateBasis {
+  double nfull[kMaxW * kMaxW];
+  int32_t cols;
+};
+
 // alpha_j == beta_i exactly when (2j+1)(W-1) == 2 K i.
 inline bool nodes_coincide(int K, int W, int j, int i) { return (2 * j + 1) * (W - 1) == 2 * K * i; }
 
@@ -39,6 +47,7 @@ long double node_gap(int K, int W, int j, int i);
 void build_encode_tables(int K, int W, EncodeTables* t);
 void build_decode_tables(int K, int W, DecodeTables* t);
 void build_locate_tables(int W, LocateTables* t);
+void build_locate_basis(int W, int M, LocateBasis* t);
 
 // The tables depend on (K, W) only and cost 10-200 us of host time to build, so each is built once per
 // process and (K, W) and then served from an immutable, mutex-protected cache.  The references stay valid
@@ -46,5 +55,6 @@ void build_locate_tables(int W, LocateTables* t);
 const EncodeTables& encode_tables(int K, int W);
 const DecodeTables& decode_tables(int K, int W);
 const LocateTables& locate_tables(int W);
+const LocateBasis& locate_basis(int W, int M);
 
 }  // namespace approxifer
