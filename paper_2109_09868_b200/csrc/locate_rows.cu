@@ -73,15 +73,13 @@ __device__ __forceinline__ int nth_set_bit(uint32_t m, int r) {
   return pos;
 }
 
-// 1/sqrt(h) for a positive, normal h: hardware seed (about 23 bits) and two Newton steps, no special cases.
-// The Givens rotations only need cs^2 + sn^2 = 1 to rounding, which this gives.
-__device__ __forceinline__ double rsqrt_pos(double h) {
+// 1/h for a positive, normal h: hardware seed (about 20 bits) and two Newton steps, no special cases.
+__device__ __forceinline__ double rcp_pos(double h) {
   double y;
-  asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(h));
-  const double hh = 0.5 * h;
-  double e = fma(-hh * y, y, 0.5);
+  asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(h));
+  double e = fma(-h, y, 1.0);
   y = fma(y, e, y);
-  e = fma(-hh * y, y, 0.5);
+  e = fma(-h, y, 1.0);
   y = fma(y, e, y);
   return y;
 }
@@ -235,11 +233,8 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
   {
     // the full-set basis, transposed and zero-padded, behind the warps' reflector scratch
     double* nft = reinterpret_cast<double*>(scratch) + kRowsWarps * M * NMAX;
-    const int dn = a.W - M;
-    for (int idx = tid; idx < (NMAX - M) * NMAX; idx += kRowsThreads) {
-      const int d = idx / NMAX, i = idx - d * NMAX;
-      nft[idx] = (d < dn && i < a.W) ? basis.nfull[i * dn + d] : 0.0;
-    }
+    // (the host lays the table out exactly as it is used here: consecutive threads copy consecutive entries)
+    for (int idx = tid; idx < (NMAX - M) * NMAX; idx += kRowsThreads) nft[idx] = basis.nft[idx];
     __syncthreads();
     double(*refl)[NMAX] = reinterpret_cast<double(*)[NMAX]>(scratch) + warp * M;
     for (int s = warp; s < ng; s += kRowsWarps) {
@@ -262,13 +257,16 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
 #pragma unroll
     for (int i = 0; i < NMAX; ++i) ysm[i * kRowsThreads] = (i < n) ? __ldg(Yc + sm.yoff[i]) : 0.f;
 
-    // upper-triangular factor R (only j >= k is ever touched) and transformed right-hand side d
-    double R[NQ][NQ], d[NQ];
+    // Square-root-free triangular factor: R = sqrt(D) U with U unit upper triangular (only j > k is ever
+    // touched) and the transformed right-hand side sqrt(D) d.  Folding a row costs two multiply-adds per
+    // entry and one reciprocal per column, no square roots, and the unknowns come out of U q = d directly.
+    double U[NQ][NQ], dg[NQ], d[NQ];
 #pragma unroll
     for (int k = 0; k < NQ; ++k) {
       d[k] = 0.0;
+      dg[k] = 0.0;
 #pragma unroll
-      for (int j = 0; j < NQ; ++j) R[k][j] = 0.0;
+      for (int j = 0; j < NQ; ++j) U[k][j] = 0.0;
     }
 
     const int rows = n - M;
@@ -293,37 +291,39 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
           row[l + 1] = fma(u1, p1.y, row[l + 1]);
         }
       }
-      // fold the equation  sum_k row[k+1] q_k = -row[0]  into (R, d) with Givens rotations
+      // fold the equation  sum_k row[k+1] q_k = -row[0]  (weight w, 1 at the start) into (D, U, d): the
+      // square-root-free form of a Givens rotation per column (Gentleman's row update)
       double rhs = -row[0];
+      double w = 1.0;
 #pragma unroll
       for (int k = 0; k < NQ; ++k) {
-        const double av = R[k][k], bv = row[k + 1];
-        const double h2 = fma(av, av, bv * bv);
-        if (h2 > 1e-290) {  // (an exactly zero column leaves the factor as it is)
-          const double rinv = rsqrt_pos(h2);
-          const double cs = av * rinv, sn = bv * rinv;
-          R[k][k] = h2 * rinv;
+        const double xk = row[k + 1];
+        const double wx = w * xk;
+        const double dn = fma(wx, xk, dg[k]);
+        if (dn > 1e-290) {  // (an exactly zero column leaves the factor as it is)
+          const double inv = rcp_pos(dn);
+          const double sb = wx * inv;
+          w *= dg[k] * inv;
+          dg[k] = dn;
 #pragma unroll
           for (int j = k + 1; j < NQ; ++j) {
-            const double rj = R[k][j], xj = row[j + 1];
-            R[k][j] = fma(cs, rj, sn * xj);
-            row[j + 1] = fma(cs, xj, -sn * rj);
+            row[j + 1] = fma(-xk, U[k][j], row[j + 1]);
+            U[k][j] = fma(sb, row[j + 1], U[k][j]);
           }
-          const double dk = d[k];
-          d[k] = fma(cs, dk, sn * rhs);
-          rhs = fma(cs, rhs, -sn * dk);
+          rhs = fma(-xk, d[k], rhs);
+          d[k] = fma(sb, rhs, d[k]);
         }
       }
     }
 
-    // back substitution; an exactly zero pivot leaves its unknown at 0
+    // back substitution (unit diagonal); a column that never received a non-zero entry keeps its unknown at 0
     double q[NQ];
 #pragma unroll
     for (int k = NQ - 1; k >= 0; --k) {
       double v = d[k];
 #pragma unroll
-      for (int j = k + 1; j < NQ; ++j) v = fma(-R[k][j], q[j], v);
-      q[k] = (R[k][k] != 0.0) ? v / R[k][k] : 0.0;
+      for (int j = k + 1; j < NQ; ++j) v = fma(-U[k][j], q[j], v);
+      q[k] = v;
     }
 
     // a_i = Q(b_i) = 1 + sum_k q_k b_i^(k+1); the E smallest |a_i| (ties to the lower worker) get a vote

@@ -78,8 +78,8 @@ void build_locate_tables(int W, LocateTables* t) {
 
 void build_locate_basis(int W, int M, LocateBasis* t) {
   std::memset(t, 0, sizeof(*t));
-  t->cols = W - M;
   if (M < 1 || M >= W) return;
+  const int P = (W + 7) / 8 * 8;
   // Householder QR of the W x M matrix [T_k(beta_i)] (Chebyshev polynomials: the same column spaces as the
   // monomials, far better conditioned), in extended precision.  Columns M .. W-1 of Q = H_0 .. H_{M-1} are
   // the basis.
@@ -114,7 +114,7 @@ void build_locate_basis(int W, int M, LocateBasis* t) {
       for (int i = k; i < W; ++i) dot += v[k][i] * q[i];
       for (int i = k; i < W; ++i) q[i] -= dot * v[k][i];
     }
-    for (int i = 0; i < W; ++i) t->nfull[i * (W - M) + d] = (double)q[i];
+    for (int i = 0; i < W; ++i) t->nft[d * P + i] = (double)q[i];
   }
 }
 

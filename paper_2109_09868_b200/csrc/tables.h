@@ -29,12 +29,13 @@ struct LocateTables {
   double beta[kMaxW];
 };
 
-// Orthonormal basis of the orthogonal complement of {polynomials of degree < M} on the FULL node set
-// beta_0 .. beta_{W-1} (all workers present): nfull[i * cols + d], cols = W - M.  The locator derives the
-// basis of a group with a few workers missing from this one instead of factorising from scratch.
+// Orthonormal basis Nf of the orthogonal complement of {polynomials of degree < M} on the FULL node set
+// beta_0 .. beta_{W-1} (all workers present), stored transposed and zero-padded the way the locator keeps it
+// in shared memory: nft[d * P + i] = Nf[i][d] for i < W, d < W - M, with P = W rounded up to a multiple of 8;
+// (P - M) * P entries are meaningful, the rest is 0.  The locator derives the basis of a group with a few
+// workers missing from this one instead of factorising from scratch.
 struct LocateBasis {
-  double nfull[kMaxW * kMaxW];
-  int32_t cols;
+  double nft[kMaxW * kMaxW];
 };
 
 // alpha_j == beta_i exactly when (2j+1)(W-1) == 2 K i.
