@@ -312,6 +312,9 @@ def other_workloads(ap, dev, peak):
     t5 = trusted.cpu().numpy().view(np.uint32)
     med, mn = time_launches(lambda: ap.approxifer_decode(p5, Yt, trusted, Yh), 3, 10)
     entry("configs[4] decode from trusted K=8 W=24 C=10 (L2-resident)", decode_bytes(w5, t5), med, mn, w5.G)
+    med, mn = time_launches(lambda: ap.approxifer_locate_decode(p5, Yt, mt, Yh), 3, 10)
+    entry("configs[4] locate + decode from trusted in one call (one kernel; predictions read once)",
+          locate_bytes(w5, m5) + 4 * w5.G * w5.K * w5.C, med, mn, w5.G)
     # workload 1: tiny, launch-latency bound
     w1 = wl.workload(1)
     p1 = ap.make_params(w1.K, w1.W)
@@ -353,6 +356,12 @@ def run_case(ap, dev, args):
             trusted = torch.empty((w.G,), dtype=torch.int32, device=dev)
             med, mn = time_launches(lambda: ap.approxifer_locate(p, Yt, mt, adv, trusted), warm, iters)
             nbytes = locate_bytes(w, m)
+        elif op == "pair":
+            adv = torch.empty((w.G, w.E), dtype=torch.int32, device=dev)
+            trusted = torch.empty((w.G,), dtype=torch.int32, device=dev)
+            Yh = torch.empty((w.G, w.K, w.C), device=dev)
+            med, mn = time_launches(lambda: ap.approxifer_locate_decode(p, Yt, mt, Yh), warm, iters)
+            nbytes = locate_bytes(w, m) + 4 * w.G * w.K * w.C
         else:
             Yh = torch.empty((w.G, w.K, w.C), device=dev)
             med, mn = time_launches(lambda: ap.approxifer_decode(p, Yt, mt, Yh), warm, iters)
@@ -414,7 +423,7 @@ def main():
     ap_.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap_.add_argument("--no-cpu", action="store_true", help="skip timing the CPU checker")
     ap_.add_argument("--groups", type=int, default=None, help="override the number of groups (profiling only)")
-    ap_.add_argument("--case", default=None, choices=["decode3", "decode4", "locate5", "decode5", "decode2", "encode3"],
+    ap_.add_argument("--case", default=None, choices=["decode3", "decode4", "locate5", "decode5", "pair5", "decode2", "encode3"],
                      help="time one kernel of another configuration alone (tuning / profiling) and print a short JSON line")
     ap_.add_argument("--dec-config", default=None, help="stages,ctas_per_sm,disable,cols,split for the wide decoder (tuning)")
     args = ap_.parse_args()
