@@ -309,6 +309,12 @@ def other_workloads(ap, dev, peak):
            "roofline": {"bound": "alu", "achieved": flops / med / 1e9, "peak": fp64_peak, "unit": "TFLOP/s",
                         "frac": flops / med / 1e9 / fp64_peak,
                         "note": "algorithmic fp64 flop of Algorithm 2's per-class least squares / time; peak = 148 SMs x 64 DFMA/clk x 2 x 1.965 GHz"}})
+    p5h = ap.make_params(w5.K, w5.W, w5.E, 2)
+    med, mn = time_launches(lambda: ap.approxifer_locate(p5h, Yt, mt, adv, trusted), 3, 10)
+    recall_h = float((adv.cpu().numpy() == adv_true).all(axis=1).mean())
+    entry("configs[4] locate, Algorithm 1's homogeneous system (|Q| = 1) per class", locate_bytes(w5, m5), med, mn, w5.G,
+          {"located_equals_injected": recall_h})
+    ap.approxifer_locate(p5, Yt, mt, adv, trusted)
     t5 = trusted.cpu().numpy().view(np.uint32)
     med, mn = time_launches(lambda: ap.approxifer_decode(p5, Yt, trusted, Yh), 3, 10)
     entry("configs[4] decode from trusted K=8 W=24 C=10 (L2-resident)", decode_bytes(w5, t5), med, mn, w5.G)
@@ -331,6 +337,8 @@ def run_case(ap, dev, args):
     op = args.case[:-1]
     w = wl.workload(cfg, args.groups)
     p = ap.make_params(w.K, w.W, w.E)
+    if op == "locateh":  # the locator with Algorithm 1's homogeneous system
+        op, p = "locate", ap.make_params(w.K, w.W, w.E, 2)
     iters = max(args.steps, 1)
     warm = max(args.warmup, 1)
     if op == "encode":
@@ -423,7 +431,7 @@ def main():
     ap_.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap_.add_argument("--no-cpu", action="store_true", help="skip timing the CPU checker")
     ap_.add_argument("--groups", type=int, default=None, help="override the number of groups (profiling only)")
-    ap_.add_argument("--case", default=None, choices=["decode3", "decode4", "locate5", "decode5", "pair5", "decode2", "encode3"],
+    ap_.add_argument("--case", default=None, choices=["decode3", "decode4", "locate5", "locateh5", "decode5", "pair5", "decode2", "encode3"],
                      help="time one kernel of another configuration alone (tuning / profiling) and print a short JSON line")
     ap_.add_argument("--dec-config", default=None, help="stages,ctas_per_sm,disable,cols,split for the wide decoder (tuning)")
     args = ap_.parse_args()

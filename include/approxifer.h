@@ -55,7 +55,7 @@ extern "C" {
 #define APPROXIFER_OK 0
 #define APPROXIFER_E_NULL (-1)  /* a required pointer is NULL */
 #define APPROXIFER_E_RANGE (-2) /* K not in 1..32, W not in 2..32, E < 0, G < 0, D < 1, D > 2^31, stride < row length */
-#define APPROXIFER_E_PARAM (-3) /* locate: E < 1 or 2(K+E) > W; unknown flag bits */
+#define APPROXIFER_E_PARAM (-3) /* locate: E < 1, 2(K+E) > W, or the homogeneous form with K+E > 10; unknown flag bits */
 #define APPROXIFER_E_CUDA (-4)  /* the CUDA runtime reported an error at launch */
 #define APPROXIFER_E_WORKSPACE (-5) /* host-buffer entry points: the device workspace cannot hold one group */
 #define APPROXIFER_E_TOO_LARGE (-6) /* approxifer_encode_host_static: the batch does not fit the built-in staging area */
@@ -63,6 +63,7 @@ extern "C" {
 /* params.flags */
 #define APPROXIFER_SIGN_RANK 0u         /* decoder sign (-1)^(rank of worker i among those used); default */
 #define APPROXIFER_SIGN_WORKER_INDEX 1u /* decoder sign (-1)^i, the decoding equation read literally */
+#define APPROXIFER_LOCATE_HOMOGENEOUS 2u /* locator: Algorithm 1's homogeneous system (|Q| = 1) instead of Q_0 = 1 */
 
 /* status[g] bits */
 #define APPROXIFER_ST_NO_WORKERS 1u             /* decode: no worker present; the group's output is zero-filled */
@@ -74,7 +75,7 @@ typedef struct approxifer_params {
   int32_t K;      /* 1..32 queries per group */
   int32_t W;      /* 2..32 workers (paper: N+1) */
   int32_t E;      /* Byzantine workers to locate; ignored by encode and decode */
-  uint32_t flags; /* APPROXIFER_SIGN_* */
+  uint32_t flags; /* APPROXIFER_SIGN_* | APPROXIFER_LOCATE_* */
 } approxifer_params;
 
 /*
@@ -128,6 +129,15 @@ int approxifer_decode(const approxifer_params* params, int64_t G, int64_t C,
  *   status        out, [G] uint32 or NULL
  * Requires E >= 1 and 2(K+E) <= W.  A group with fewer than 2(K+E) workers
  * present gets adv = -1, trusted_mask = mask and ST_LOCATE_UNDERDETERMINED.
+ *
+ * With APPROXIFER_LOCATE_HOMOGENEOUS in params.flags the per-class step is
+ * Algorithm 1 as printed (Section 3, "Rational Interpolation with Erroneous
+ * Evaluations"): Q(x) = sum_{k<K+E} Q_k x^k with Q_0 free, and the homogeneous
+ * system P(beta_i) = y_i Q(beta_i) is solved in the least-squares sense over
+ * all P and over Q with sum_k Q_k^2 = 1 (the smallest singular direction).
+ * Selection, vote, outputs and status bits are the same.  This form has no
+ * special case at a node equal to 0 (odd W), where Q_0 = 1 pins a_i to 1.
+ * Available for K+E <= 10; APPROXIFER_E_PARAM otherwise.
  */
 int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C,
                       const float* Yt, int64_t yt_gstride, int64_t yt_rstride,

@@ -18,7 +18,7 @@ namespace {
 int check_kw(const approxifer_params* p) {
   if (p == nullptr) return APPROXIFER_E_NULL;
   if (p->K < 1 || p->K > APPROXIFER_MAX_K || p->W < 2 || p->W > APPROXIFER_MAX_W) return APPROXIFER_E_RANGE;
-  if (p->flags & ~APPROXIFER_SIGN_WORKER_INDEX) return APPROXIFER_E_PARAM;
+  if (p->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS)) return APPROXIFER_E_PARAM;
   return APPROXIFER_OK;
 }
 
@@ -73,11 +73,12 @@ int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C, con
   if (rc) return rc;
   if (params->E < 0) return APPROXIFER_E_RANGE;
   if (params->E < 1 || 2 * (params->K + params->E) > params->W) return APPROXIFER_E_PARAM;
+  if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateRowsMaxM) return APPROXIFER_E_PARAM;
   if ((rc = check_layout(G, C, yt_rstride))) return rc;
   if (yt_gstride < 0) return APPROXIFER_E_RANGE;
   if (G == 0) return APPROXIFER_OK;
   if (Yt == nullptr || mask == nullptr || adv == nullptr || trusted_mask == nullptr) return APPROXIFER_E_NULL;
-  LocateArgs a{Yt, mask, adv, trusted_mask, status, yt_gstride, yt_rstride, G, C, params->K, params->W, params->E};
+  LocateArgs a{Yt, mask, adv, trusted_mask, status, yt_gstride, yt_rstride, G, C, params->K, params->W, params->E, params->flags};
   return from_cuda(launch_locate(a, static_cast<cudaStream_t>(cuda_stream)));
 }
 

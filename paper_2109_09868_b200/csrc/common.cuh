@@ -15,6 +15,7 @@ constexpr uint32_t kStLocateUnderdetermined = 4u;
 constexpr uint32_t kStNonfinite = 8u;
 
 constexpr uint32_t kFlagSignWorkerIndex = 1u;
+constexpr uint32_t kFlagLocateHomogeneous = 2u;
 
 struct EncodeArgs {
   const float* X;
@@ -45,6 +46,7 @@ struct LocateArgs {
   int64_t y_gs, y_rs;
   int64_t G, C;
   int32_t K, W, E;
+  uint32_t flags;
 };
 
 // Each returns a cudaError_t from the launch (cudaSuccess if nothing to do).

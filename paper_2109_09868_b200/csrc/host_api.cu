@@ -151,6 +151,8 @@ int approxifer_locate_host(const approxifer_params* params, int64_t G, int64_t C
   if (params->K < 1 || params->K > APPROXIFER_MAX_K || params->W < 2 || params->W > APPROXIFER_MAX_W || params->E < 0)
     return APPROXIFER_E_RANGE;
   if (params->E < 1 || 2 * (params->K + params->E) > params->W) return APPROXIFER_E_PARAM;
+  if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS)) return APPROXIFER_E_PARAM;
+  if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateRowsMaxM) return APPROXIFER_E_PARAM;
   if (G < 0 || C < 1 || C > (int64_t(1) << 31)) return APPROXIFER_E_RANGE;
   if (G == 0) return APPROXIFER_OK;
   if (hYt == nullptr || hmask == nullptr || hadv == nullptr || htrusted == nullptr || workspace == nullptr ||
@@ -178,7 +180,7 @@ int approxifer_locate_host(const approxifer_params* params, int64_t G, int64_t C
     uint32_t* dst = reinterpret_cast<uint32_t*>(slice + off);
     if (cudaMemcpyAsync(dYt, hYt + g0 * W * C, (size_t)ng * W * C * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return APPROXIFER_E_CUDA;
     if (cudaMemcpyAsync(dmask, hmask + g0, (size_t)ng * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return APPROXIFER_E_CUDA;
-    LocateArgs a{dYt, dmask, dadv, dtr, dst, (int64_t)W * C, C, ng, C, K, W, E};
+    LocateArgs a{dYt, dmask, dadv, dtr, dst, (int64_t)W * C, C, ng, C, K, W, E, params->flags};
     if (launch_locate(a, st) != cudaSuccess) return APPROXIFER_E_CUDA;
     if (cudaMemcpyAsync(hadv + g0 * E, dadv, (size_t)ng * E * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return APPROXIFER_E_CUDA;
     if (cudaMemcpyAsync(htrusted + g0, dtr, (size_t)ng * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return APPROXIFER_E_CUDA;

@@ -272,7 +272,8 @@ cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   const LocateTables& tab = locate_tables(a.W);
   const int m = a.K + a.E;
-  if (m <= kLocateRowsMaxM && !g_force_warp_kernel) return launch_locate_rows(a, tab, stream);
+  // (the homogeneous form exists in the thread-per-class kernel only; the entry point has checked K+E)
+  if (m <= kLocateRowsMaxM && (!g_force_warp_kernel || (a.flags & kFlagLocateHomogeneous))) return launch_locate_rows(a, tab, stream);
   if (a.W <= 8) return dispatch_m<8>(m, a, tab, stream);
   if (a.W <= 16) return dispatch_m<16>(m, a, tab, stream);
   if (a.W <= 24) return dispatch_m<24>(m, a, tab, stream);

@@ -210,7 +210,9 @@ __device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double 
 }
 
 
-template <int NMAX, int M>
+// HOMOG: Algorithm 1's homogeneous system (Q_0 free) solved in the least-squares sense with |Q| = 1, instead of
+// Algorithm 2's normalisation Q_0 = 1; everything else (basis, rows, selection, vote) is shared.
+template <int NMAX, int M, bool HOMOG>
 __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __grid_constant__ LocateArgs a,
                                                                       const __grid_constant__ LocateTables tab,
                                                                       const __grid_constant__ LocateBasis basis,
@@ -260,14 +262,18 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
     // Square-root-free triangular factor: R = sqrt(D) U with U unit upper triangular (only j > k is ever
     // touched) and the transformed right-hand side sqrt(D) d.  Folding a row costs two multiply-adds per
     // entry and one reciprocal per column, no square roots, and the unknowns come out of U q = d directly.
-    double U[NQ][NQ], dg[NQ], d[NQ];
+    // (homogeneous form: column 0 is one more unknown instead of the right-hand side, NC = M columns)
+    constexpr int NC = HOMOG ? M : NQ;   // columns of the factor
+    constexpr int C0 = HOMOG ? 0 : 1;    // row[] index of the factor's first column
+    double U[NC][NC], dg[NC], d[NQ];
 #pragma unroll
-    for (int k = 0; k < NQ; ++k) {
-      d[k] = 0.0;
+    for (int k = 0; k < NC; ++k) {
       dg[k] = 0.0;
 #pragma unroll
-      for (int j = 0; j < NQ; ++j) U[k][j] = 0.0;
+      for (int j = 0; j < NC; ++j) U[k][j] = 0.0;
     }
+#pragma unroll
+    for (int k = 0; k < NQ; ++k) d[k] = 0.0;
 
     const int rows = n - M;
 #pragma unroll 1
@@ -296,8 +302,8 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
       double rhs = -row[0];
       double w = 1.0;
 #pragma unroll
-      for (int k = 0; k < NQ; ++k) {
-        const double xk = row[k + 1];
+      for (int k = 0; k < NC; ++k) {
+        const double xk = row[k + C0];
         const double wx = w * xk;
         const double dn = fma(wx, xk, dg[k]);
         if (dn > 1e-290) {  // (an exactly zero column leaves the factor as it is)
@@ -306,24 +312,73 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
           w *= dg[k] * inv;
           dg[k] = dn;
 #pragma unroll
-          for (int j = k + 1; j < NQ; ++j) {
-            row[j + 1] = fma(-xk, U[k][j], row[j + 1]);
-            U[k][j] = fma(sb, row[j + 1], U[k][j]);
+          for (int j = k + 1; j < NC; ++j) {
+            row[j + C0] = fma(-xk, U[k][j], row[j + C0]);
+            U[k][j] = fma(sb, row[j + C0], U[k][j]);
           }
-          rhs = fma(-xk, d[k], rhs);
-          d[k] = fma(sb, rhs, d[k]);
+          if constexpr (!HOMOG) {
+            rhs = fma(-xk, d[k], rhs);
+            d[k] = fma(sb, rhs, d[k]);
+          }
         }
       }
     }
 
-    // back substitution (unit diagonal); a column that never received a non-zero entry keeps its unknown at 0
-    double q[NQ];
+    // q[k] = Q_{k+1} (Algorithm 2) or Q_k (homogeneous form)
+    double q[NC];
+    if constexpr (!HOMOG) {
+      // back substitution (unit diagonal); a column that never received a non-zero entry keeps its unknown at 0
 #pragma unroll
-    for (int k = NQ - 1; k >= 0; --k) {
-      double v = d[k];
+      for (int k = NQ - 1; k >= 0; --k) {
+        double v = d[k];
 #pragma unroll
-      for (int j = k + 1; j < NQ; ++j) v = fma(-U[k][j], q[j], v);
-      q[k] = v;
+        for (int j = k + 1; j < NQ; ++j) v = fma(-U[k][j], q[j], v);
+        q[k] = v;
+      }
+    } else {
+      // The unit vector q that minimises |R q|, R^T R = U^T D U: inverse iteration (two unit-triangular solves
+      // and a diagonal scaling per step), stopped when the direction no longer moves, then two more steps.
+      double dmax = 0.0;
+#pragma unroll
+      for (int k = 0; k < NC; ++k) dmax = fmax(dmax, dg[k]);
+      const double floor_d = fmax(dmax * 1e-30, 1e-300);
+#pragma unroll
+      for (int k = 0; k < NC; ++k) dg[k] = 1.0 / fmax(dg[k], floor_d);  // from here on: 1/D (floored)
+#pragma unroll
+      for (int k = 0; k < NC; ++k) q[k] = 0.3 + 0.07 * k;
+      int extra = 2;
+#pragma unroll 1
+      for (int it = 0; it < 300 && extra >= 0; ++it) {
+        double t[NC];
+#pragma unroll
+        for (int k = 0; k < NC; ++k) {  // U^T t = q
+          double v = q[k];
+#pragma unroll
+          for (int j = 0; j < k; ++j) v = fma(-U[j][k], t[j], v);
+          t[k] = v;
+        }
+#pragma unroll
+        for (int k = 0; k < NC; ++k) t[k] *= dg[k];
+#pragma unroll
+        for (int k = NC - 1; k >= 0; --k) {  // U z = t, in place
+          double v = t[k];
+#pragma unroll
+          for (int j = k + 1; j < NC; ++j) v = fma(-U[k][j], t[j], v);
+          t[k] = v;
+        }
+        double n2 = 0.0, dot = 0.0;
+#pragma unroll
+        for (int k = 0; k < NC; ++k) {
+          n2 = fma(t[k], t[k], n2);
+          dot = fma(t[k], q[k], dot);
+        }
+        const double inv = rsqrt(n2);
+        // q is a unit vector after the first step; |dot| * inv = |cos| of the angle between the two iterates
+        const bool settled = it > 0 && (1.0 - fabs(dot) * inv) <= 4e-16;
+        if (settled || extra < 2) --extra;
+#pragma unroll
+        for (int k = 0; k < NC; ++k) q[k] = t[k] * inv;
+      }
     }
 
     // a_i = Q(b_i) = 1 + sum_k q_k b_i^(k+1); the E smallest |a_i| (ties to the lower worker) get a vote
@@ -332,10 +387,10 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
 #pragma unroll
     for (int i = 0; i < NMAX; ++i) {
       const double b = sm.xs[i];
-      double h = q[NQ - 1];
+      double h = q[NC - 1];
 #pragma unroll
-      for (int k = NQ - 2; k >= 0; --k) h = fma(h, b, q[k]);
-      const double av = fma(h, b, 1.0);
+      for (int k = NC - 2; k >= 0; --k) h = fma(h, b, q[k]);
+      const double av = HOMOG ? h : fma(h, b, 1.0);
       const bool fin = isfinite(av);
       mag[i] = fin ? fabs(av) : INFINITY;
       nonfinite |= (i < n) && !fin;
@@ -408,15 +463,19 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
   while (gpb > 1 && gpb * per_group + y_bytes > 74 * 1024) --gpb;
   if (gpb > a.G) gpb = a.G;
   const size_t smem = (size_t)gpb * per_group + y_bytes;
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(locate_rows_kernel<NMAX, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-  }
   const int64_t blocks = (a.G + gpb - 1) / gpb;
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-  locate_rows_kernel<NMAX, M><<<(unsigned)blocks, kRowsThreads, smem, stream>>>(a, tab, locate_basis(a.W, M), (int)gpb);
-  count_launch();
-  return cudaGetLastError();
+  auto run = [&](auto kernel) -> cudaError_t {
+    if (smem > 48 * 1024) {
+      cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
+    kernel<<<(unsigned)blocks, kRowsThreads, smem, stream>>>(a, tab, locate_basis(a.W, M), (int)gpb);
+    count_launch();
+    return cudaGetLastError();
+  };
+  if (a.flags & kFlagLocateHomogeneous) return run(locate_rows_kernel<NMAX, M, true>);
+  return run(locate_rows_kernel<NMAX, M, false>);
 }
 
 template <int NMAX, int M = 2>

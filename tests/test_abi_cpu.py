@@ -56,7 +56,7 @@ def test_encode_argument_errors_are_reported_on_the_host():
     assert _encode_rc(4, 5, 1, 8, orr=4) == binding.E_RANGE
     assert _encode_rc(4, 5, 1, 8, x=None) == binding.E_NULL
     assert _encode_rc(4, 5, 1, 8, xt=None) == binding.E_NULL
-    assert _encode_rc(4, 5, 1, 8, flags=2) == binding.E_PARAM
+    assert _encode_rc(4, 5, 1, 8, flags=4) == binding.E_PARAM  # unknown flag bit
     assert _encode_rc(4, 5, 0, 8, x=None, xt=None) == binding.OK  # G = 0: valid no-op
     assert ap.load().approxifer_encode(None, 1, 8, 1, 32, 8, 1, 40, 8, None) == binding.E_NULL
 
@@ -74,6 +74,10 @@ def test_decode_and_locate_argument_errors():
         assert rc == want, (K, W, E)
     q = ap.make_params(8, 24, 2)
     assert lib.approxifer_locate(ctypes.byref(q), 1, 10, 1, 240, 10, 1, None, 1, None, None) == binding.E_NULL
+    # the homogeneous form of the locator exists for K+E <= 10
+    for (K, W, E, want) in [(8, 24, 2, binding.OK), (9, 32, 2, binding.E_PARAM), (12, 32, 2, binding.E_PARAM)]:
+        q = ap.make_params(K, W, E, binding.LOCATE_HOMOGENEOUS)
+        assert lib.approxifer_locate(ctypes.byref(q), 0, 10, None, W * 10, 10, None, None, None, None, None) == want
 
 
 def test_binding_refuses_cpu_tensors():

@@ -99,8 +99,8 @@ def _linear_predictions(K, W, G, C, rng, d_in=6):
 
 @pytest.mark.parametrize("K,E,S", [(2, 1, 0), (3, 2, 1), (4, 1, 2), (8, 2, 2), (6, 3, 1), (5, 1, 0)])
 def test_locates_injected_errors_for_a_linear_model(K, E, S):
-    """Theorem 1 through the whole procedure.  Unlike Algorithm 2 (Q_0 = 1) the homogeneous form can
-    flag a worker whose node is 0, so an odd number of workers is as good as an even one."""
+    """Theorem 1 through the whole procedure.  Unlike Algorithm 2 (Q_0 = 1, which pins a_i = 1 at a node
+    equal to 0) the homogeneous form has no special node, so an odd number of workers is as good as an even one."""
     rng = np.random.default_rng(300 + K * 10 + E)
     W = 2 * (K + E) + S
     G, C = 30, 4
