@@ -140,3 +140,27 @@ def test_workload5_full_size_homogeneous_form():
     assert ref["min_gap"].min() > 1.5 and np.all(ref["vote_margin"] > 0) and np.all(ref["status"] == 0)
     np.testing.assert_array_equal(adv[sel], ref["adv"])
     np.testing.assert_array_equal(trusted[sel], ref["trusted"])
+
+
+def test_homogeneous_flag_through_the_one_call_and_host_buffer_entry_points():
+    """approxifer_locate_decode and approxifer_locate_host honour the flag: same sets as approxifer_locate with
+    it, and the decoded predictions equal a separate decode from those trusted workers (the decoder ignores the flag)."""
+    K, E, S, W, G, C = 4, 2, 1, 13, 70, 6
+    Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=5)
+    p = ap.make_params(K, W, E, binding.LOCATE_HOMOGENEOUS)
+    Yd, md = Yt.to(dev()), ap.mask_tensor(mask)
+    adv, trusted = ap.approxifer_locate(p, Yd, md)
+    Yh, adv1, trusted1 = ap.approxifer_locate_decode(p, Yd, md)
+    assert torch.equal(adv, adv1) and torch.equal(trusted, trusted1)
+    assert torch.equal(Yh, ap.approxifer_decode(ap.make_params(K, W), Yd, trusted))
+    np.testing.assert_array_equal(adv.cpu().numpy(), truth)
+    hYt = Yt.pin_memory()
+    hmask = torch.from_numpy(mask.view(np.int32).copy()).pin_memory()
+    hadv = torch.empty((G, E), dtype=torch.int32).pin_memory()
+    htr = torch.empty((G,), dtype=torch.int32).pin_memory()
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device=dev())
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    ap.approxifer_locate_host(p, hYt, hmask, hadv, htr, ws, streams)
+    for st in streams:
+        st.synchronize()
+    assert torch.equal(hadv, adv.cpu()) and torch.equal(htr, trusted.cpu())
