@@ -62,6 +62,11 @@ cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, c
 void decode_staged_config(int stages, int ctas_per_sm, int disable, int cols, int split);
 cudaError_t read_decode_wait_timeouts(unsigned int* out);
 
+// Short-payload decoder (C <= 32, dense buffers); see decode_small.cu.
+bool decode_small_eligible(const DecodeArgs& a);
+cudaError_t launch_decode_small(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream);
+void decode_small_config(int disable);
+
 // Thread-per-class locator for K+E <= kLocateRowsMaxM (locate_rows.cu); the warp-per-group kernel covers the rest.
 constexpr int kLocateRowsMaxM = 10;
 cudaError_t launch_locate_rows(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream);

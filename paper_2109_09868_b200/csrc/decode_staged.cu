@@ -421,6 +421,7 @@ void decode_staged_config(int stages, int ctas_per_sm, int disable, int cols, in
   g_cfg_stages = stages;
   g_cfg_ctas_per_sm = ctas_per_sm;
   g_cfg_disable = disable;
+  decode_small_config(disable);
   g_cfg_cols = cols;
 }
 

@@ -12,6 +12,7 @@ import torch
 
 import oracle
 import paper_2109_09868_b200 as ap
+from paper_2109_09868_b200 import binding
 from paper_2109_09868_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -416,6 +417,39 @@ def test_staged_and_register_decoders_agree_bitwise_on_sums_order():
     finally:
         ap.debug_decode_config(0, 0, 0)
     assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("K,W,C,G", [(8, 12, 10, 1000), (8, 24, 10, 333), (4, 5, 10, 7), (3, 7, 9, 130), (1, 2, 1, 50),
+                                     (32, 32, 32, 21), (16, 24, 31, 64), (2, 5, 2, 257), (12, 20, 17, 90), (5, 9, 4, 3)])
+def test_short_payload_decoder_against_oracle_and_register_decoder(K, W, C, G):
+    """Dense buffers with at most 32 classes take the thread-per-query kernel.  It adds the same terms in the same
+    order as the thread-per-class kernel: equal to the last bit, absent rows (NaN here) never used, both sign
+    rules, coincident nodes ((K, W) = (3, 7), (1, 2) and (2, 5) have them), group counts that leave a ragged last CTA."""
+    rng = np.random.default_rng(K * 100 + C)
+    Yt = torch.randn((G, W, C), generator=torch.Generator().manual_seed(C))
+    mask = random_masks(W, G, rng, min_present=0)
+    mask[0] = 0
+    dirty = Yt.clone()
+    for gi in range(G):
+        for i in range(W):
+            if not (int(mask[gi]) >> i) & 1:
+                dirty[gi, i] = float("nan")
+    for flags in (0, binding.SIGN_WORKER_INDEX):
+        p = ap.make_params(K, W, 0, flags)
+        n_used = torch.empty(G, dtype=torch.int32, device=dev())
+        status = torch.empty(G, dtype=torch.int32, device=dev())
+        guard = torch.full((G * K * C + 64,), CANARY, device=dev())
+        Yh = guard[32: 32 + G * K * C].view(G, K, C)
+        ap.approxifer_decode(p, dirty.to(dev()), ap.mask_tensor(mask), Yh, n_used=n_used, status=status)
+        if flags == 0:  # (the literal sign has poles: on arbitrary masks a denominator can vanish, see pin P9)
+            check_decode(K, W, Yt, mask, Yh, n_used, status, flags)
+        assert bool((guard[:32] == CANARY).all()) and bool((guard[32 + G * K * C:] == CANARY).all())
+        try:
+            ap.debug_decode_config(0, 0, 1)
+            ref = ap.approxifer_decode(p, dirty.to(dev()), ap.mask_tensor(mask))
+        finally:
+            ap.debug_decode_config(0, 0, 0)
+        assert torch.equal(Yh.contiguous().view(torch.int32), ref.view(torch.int32))  # bit patterns: inf/NaN included
 
 
 def test_worker_major_layouts_for_decode_and_locate():
