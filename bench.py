@@ -319,7 +319,7 @@ def other_workloads(ap, dev, peak):
     med, mn = time_launches(lambda: ap.approxifer_decode(p5, Yt, trusted, Yh), 3, 10)
     entry("configs[4] decode from trusted K=8 W=24 C=10 (L2-resident)", decode_bytes(w5, t5), med, mn, w5.G)
     med, mn = time_launches(lambda: ap.approxifer_locate_decode(p5, Yt, mt, Yh), 3, 10)
-    entry("configs[4] locate + decode from trusted in one call (one kernel; predictions read once)",
+    entry("configs[4] locate + decode from trusted through approxifer_locate_decode (two launches)",
           locate_bytes(w5, m5) + 4 * w5.G * w5.K * w5.C, med, mn, w5.G)
     # workload 1: tiny, launch-latency bound
     w1 = wl.workload(1)
