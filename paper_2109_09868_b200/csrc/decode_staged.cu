@@ -401,13 +401,41 @@ cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t
   return cudaGetLastError();
 }
 
+// Columns per work item.  Long contiguous pieces are what HBM likes: with 256 columns an item of workload 4
+// (rows of 250 float4) is whole rows -- one 4000-byte copy per present worker instead of two copies of about 2 KB
+// issued by different CTAs at different times -- and the kernel runs 6 % faster (one CTA of 16 compute warps per
+// SM instead of two of 8).  256 is taken when a two-slot ring of such items fits in shared memory and wastes no
+// more threads on the ragged last tile than 128 would.
+template <int KT, int SPLIT>
+bool fits_256(const DecodeArgs& a) {
+  if (SPLIT != 2 || KT > 8) return false;  // 544 threads leave 112 registers each: enough for 8 queries per thread
+  int dev = 0, smem_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
+    return false;
+  return (int64_t)slots_off(a.W, a.K) + 2 * (int64_t)slot_bytes(a.W, KT, SPLIT, 256) + 1024 <= smem_sm;
+}
+
+template <int KT, int SPLIT>
+int auto_cols(const DecodeArgs& a) {
+  if (!fits_256<KT, SPLIT>(a)) return 128;
+  const int64_t Cv = a.C / 4;
+  const int64_t waste256 = (Cv + 255) / 256 * 256 - Cv, waste128 = (Cv + 127) / 128 * 128 - Cv;
+  return waste256 <= waste128 ? 256 : 128;
+}
+
 template <int SPLIT, int KT = 1>
 cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream) {
   if constexpr (KT > kMaxK / SPLIT) {
     return cudaErrorInvalidValue;
   } else {
     if (kt == KT) {
-      if (g_cfg_cols == 64) return launch_kt<KT, 64, SPLIT>(a, tab, stream);
+      int cols = g_cfg_cols ? g_cfg_cols : auto_cols<KT, SPLIT>(a);
+      if (cols == 256 && !fits_256<KT, SPLIT>(a)) cols = 128;  // (a forced setting that cannot be honoured)
+      if (cols == 64) return launch_kt<KT, 64, SPLIT>(a, tab, stream);
+      if constexpr (SPLIT == 2 && KT <= 8) {
+        if (cols == 256) return launch_kt<KT, 256, SPLIT>(a, tab, stream);
+      }
       return launch_kt<KT, 128, SPLIT>(a, tab, stream);
     }
     return dispatch_kt<SPLIT, KT + 1>(kt, a, tab, stream);

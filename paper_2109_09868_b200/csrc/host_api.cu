@@ -96,13 +96,15 @@ int approxifer_decode_host(const approxifer_params* params, int64_t G, int64_t C
                            void* const* cuda_streams, int n_streams) {
   if (params == nullptr) return APPROXIFER_E_NULL;
   if (params->K < 1 || params->K > APPROXIFER_MAX_K || params->W < 2 || params->W > APPROXIFER_MAX_W) return APPROXIFER_E_RANGE;
-  if (params->flags & ~APPROXIFER_SIGN_WORKER_INDEX) return APPROXIFER_E_PARAM;
+  if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS)) return APPROXIFER_E_PARAM;
   if (G < 0 || C < 1 || C > (int64_t(1) << 31)) return APPROXIFER_E_RANGE;
   if (G == 0) return APPROXIFER_OK;
   if (hYt == nullptr || hmask == nullptr || hYhat == nullptr || workspace == nullptr || cuda_streams == nullptr)
     return APPROXIFER_E_NULL;
   const int K = params->K, W = params->W;
-  const int64_t Cp = (C + 3) & ~int64_t(3);
+  // staged rows are padded to whole float4s for the 128-bit kernels; short rows (C <= 32) stay dense, which is
+  // what the short-payload decoder takes and turns both copies into plain contiguous ones
+  const int64_t Cp = (C <= 32) ? C : ((C + 3) & ~int64_t(3));
   const size_t in_g = (size_t)W * Cp * 4, out_g = (size_t)K * Cp * 4, small_g = 12;  // mask, n_used, status
   ChunkPlan plan;
   int rc = plan_chunks(G, in_g + out_g + small_g, 1280, workspace_bytes, n_streams, &plan);
