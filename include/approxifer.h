@@ -241,8 +241,9 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
  * with bulk asynchronous copies.  stages: 0 (as many as fit, at most 4) or an
  * upper bound >= 2 on the ring depth; ctas_per_sm: 0 (automatic) or an upper
  * bound; disable != 0 routes every decode through the register-staged kernel;
- * cols: 0 (automatic), 64, 128 or 256 (with split 2 only) 16-byte columns per work item; split: 0
- * (automatic), 2 or 4 thread groups sharing the K queries of a column.
+ * cols: 0 (automatic), 64, 128 or 256 16-byte columns per work item (256 needs split 1 or 2 and a
+ * ring that fits in shared memory, else 128 is used); split: 0 (automatic), 1 (K <= 16, 256 columns), 2 or 4
+ * thread groups sharing the K queries of a column.
  * Process-wide, not thread-safe; results are bit-identical for every setting.
  */
 int approxifer_debug_decode_config(int stages, int ctas_per_sm, int disable, int cols, int split);

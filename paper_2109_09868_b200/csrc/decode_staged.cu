@@ -401,6 +401,8 @@ cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t
   return cudaGetLastError();
 }
 
+constexpr int kWholeMaxK = 16;  // most queries one thread forms (SPLIT = 1)
+
 // Columns per work item.  Long contiguous pieces are what HBM likes: with 256 columns an item of workload 4
 // (rows of 250 float4) is whole rows -- one 4000-byte copy per present worker instead of two copies of about 2 KB
 // issued by different CTAs at different times -- and the kernel runs 6 % faster (one CTA of 16 compute warps per
@@ -408,7 +410,9 @@ cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t
 // more threads on the ragged last tile than 128 would.
 template <int KT, int SPLIT>
 bool fits_256(const DecodeArgs& a) {
-  if (SPLIT != 2 || KT > 8) return false;  // 544 threads leave 112 registers each: enough for 8 queries per thread
+  // 544 threads (two thread groups) leave 112 registers each: enough for 8 queries per thread; a single thread
+  // group of 256 carries up to 16
+  if (SPLIT == 4 || (SPLIT == 2 && KT > 8) || (SPLIT == 1 && KT > kWholeMaxK)) return false;
   int dev = 0, smem_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
@@ -436,6 +440,7 @@ cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cu
       if constexpr (SPLIT == 2 && KT <= 8) {
         if (cols == 256) return launch_kt<KT, 256, SPLIT>(a, tab, stream);
       }
+      if constexpr (SPLIT == 1) return launch_kt<KT, 256, 1>(a, tab, stream);  // (the only single-group shape)
       return launch_kt<KT, 128, SPLIT>(a, tab, stream);
     }
     return dispatch_kt<SPLIT, KT + 1>(kt, a, tab, stream);
@@ -466,7 +471,31 @@ bool decode_staged_eligible(const DecodeArgs& a) {
   return true;
 }
 
+// One thread group forming all K queries of a column, 256-column items: the fewest shared-memory reads and
+// register moves per multiply-add (each payload word is fetched and duplicated once, not once per thread group).
+// Under the power cap that a long run of this kernel hits, it sustains 6.2 ms on workload 4 where two groups of
+// 8 queries sustain 6.4 ms (both 5.7 ms while the clocks last).
+template <int KT = 1>
+cudaError_t dispatch_whole(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream, bool* taken) {
+  if constexpr (KT > kWholeMaxK) {
+    *taken = false;
+    return cudaSuccess;
+  } else {
+    if (a.K == KT) {
+      const int64_t Cv = a.C / 4;
+      const int64_t waste256 = (Cv + 255) / 256 * 256 - Cv, waste128 = (Cv + 127) / 128 * 128 - Cv;
+      const bool want = g_cfg_split == 1 || (g_cfg_split == 0 && (g_cfg_cols == 0 || g_cfg_cols == 256) && waste256 <= waste128);
+      *taken = want && fits_256<KT, 1>(a);
+      return *taken ? launch_kt<KT, 256, 1>(a, tab, stream) : cudaSuccess;
+    }
+    return dispatch_whole<KT + 1>(a, tab, stream, taken);
+  }
+}
+
 cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream) {
+  bool taken = false;
+  const cudaError_t e = dispatch_whole<>(a, tab, stream, &taken);
+  if (taken) return e;
   if (g_cfg_split == 4) return dispatch_kt<4>((a.K + 3) / 4, a, tab, stream);
   return dispatch_kt<2>((a.K + 1) / 2, a, tab, stream);
 }

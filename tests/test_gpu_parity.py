@@ -372,7 +372,7 @@ STAGED_SHAPES = [
 
 
 @pytest.mark.parametrize("stages,ctas,cols,split", [(0, 0, 0, 0), (2, 0, 128, 2), (3, 1, 128, 4), (4, 1, 64, 2), (2, 4, 64, 4), (0, 2, 64, 4),
-                                                        (0, 0, 256, 2), (2, 1, 256, 0), (0, 0, 128, 0)])
+                                                        (0, 0, 256, 2), (2, 1, 256, 0), (0, 0, 128, 0), (0, 0, 0, 1), (0, 0, 0, 2)])
 def test_staged_decoder_matches_oracle_in_every_configuration(stages, ctas, cols, split):
     try:
         ap.debug_decode_config(stages, ctas, 0, cols, split)
