@@ -1,5 +1,6 @@
 """Algorithm 1 of ApproxIFER (arXiv 2109.09868, Section 3, "Rational Interpolation with
-Erroneous Evaluations") in its homogeneous form, in numpy fp64.
+Erroneous Evaluations") in its homogeneous form, and Algorithm 3 (Appendix A: the rational function
+itself, P / Q) at the end of the file, in numpy fp64.
 
 TEST INFRASTRUCTURE ONLY, like the rest of this package: the product never imports it.
 
@@ -102,3 +103,52 @@ def locate_homogeneous(K: int, W: int, E: int, Yt, mask):
         trusted[g] = mk & ~bits
     return dict(adv=adv, trusted=trusted, status=status, min_gap=min_gap, vote_margin=margin,
                 sigma_ratio=sigma_ratio)
+
+
+# ---------------------------------------------------------------------------------------------
+# Algorithm 3 (Appendix A, "BW-type rational interpolation in presence of errors")
+# ---------------------------------------------------------------------------------------------
+
+def rational_class(m: int, xs, y):
+    """Step 1 of Algorithm 3 for one scalar sequence: polynomials P, Q of degree < m with
+    P(x_i) = y_i Q(x_i) on the available nodes, solved as Algorithm 2 solves the same system
+    (Q_0 = 1, ordinary least squares).  Returns (P, Q) as coefficient arrays, Q[0] = 1."""
+    xs = np.asarray(xs, dtype=np.float64)
+    y = np.asarray(y, dtype=np.float64)
+    V = np.vander(xs, m, increasing=True)
+    A = np.hstack([V, -y[:, None] * V[:, 1:]])
+    x, *_ = np.linalg.lstsq(A, y, rcond=None)
+    return x[:m].copy(), np.concatenate([[1.0], x[m:]])
+
+
+def decode_rational(K: int, W: int, E: int, Yt, mask, alpha_nodes):
+    """Algorithm 3 per group and class, then Step 2: r = P / Q evaluated at the K nodes alpha_j.
+
+    Yt float32 [G][W][C], mask uint32 [G], alpha_nodes = oracle.alpha(K).  Returns dict(Yhat float64
+    [G][K][C] (0 where nothing was computed), status uint32 [G] (ST_LOCATE_UNDERDETERMINED for fewer
+    than 2(K+E) workers), q_min [G] = min over classes and j of |Q(alpha_j)| / max_i |Q(beta_i)|, a
+    measure of how close a pole of r comes to an output node)."""
+    Yt = np.asarray(Yt)
+    G, _, C = Yt.shape
+    mask = np.asarray(mask, dtype=np.uint32)
+    m = K + E
+    be = beta(W)
+    al = np.asarray(alpha_nodes, dtype=np.float64)
+    Va = np.vander(al, m, increasing=True)
+    wmask = 0xFFFFFFFF if W >= 32 else (1 << W) - 1
+    out = np.zeros((G, K, C))
+    status = np.zeros(G, dtype=np.uint32)
+    q_min = np.full(G, np.inf)
+    for g in range(G):
+        F = compact(W, int(mask[g]) & wmask)
+        if len(F) < 2 * m:
+            status[g] |= ST_LOCATE_UNDERDETERMINED
+            continue
+        xs = be[F]
+        Vb = np.vander(xs, m, increasing=True)
+        for c in range(C):
+            P, Q = rational_class(m, xs, Yt[g, F, c].astype(np.float64))
+            qa = Va @ Q
+            out[g, :, c] = (Va @ P) / qa
+            q_min[g] = min(q_min[g], np.abs(qa).min() / np.abs(Vb @ Q).max())
+    return dict(Yhat=out, status=status, q_min=q_min)
