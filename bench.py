@@ -314,6 +314,9 @@ def other_workloads(ap, dev, peak):
     recall_h = float((adv.cpu().numpy() == adv_true).all(axis=1).mean())
     entry("configs[4] locate, Algorithm 1's homogeneous system (|Q| = 1) per class", locate_bytes(w5, m5), med, mn, w5.G,
           {"located_equals_injected": recall_h})
+    med, mn = time_launches(lambda: ap.approxifer_decode_rational(p5, Yt, mt, Yh), 3, 10)
+    entry("configs[4] rational decoding (Algorithm 3: P/Q at the alpha nodes, nothing located)",
+          locate_bytes(w5, m5) + 4 * w5.G * w5.K * w5.C, med, mn, w5.G)
     ap.approxifer_locate(p5, Yt, mt, adv, trusted)
     t5 = trusted.cpu().numpy().view(np.uint32)
     med, mn = time_launches(lambda: ap.approxifer_decode(p5, Yt, trusted, Yh), 3, 10)
@@ -364,6 +367,10 @@ def run_case(ap, dev, args):
             trusted = torch.empty((w.G,), dtype=torch.int32, device=dev)
             med, mn = time_launches(lambda: ap.approxifer_locate(p, Yt, mt, adv, trusted), warm, iters)
             nbytes = locate_bytes(w, m)
+        elif op == "rational":  # Algorithm 3: P/Q at the alpha nodes
+            Yh = torch.empty((w.G, w.K, w.C), device=dev)
+            med, mn = time_launches(lambda: ap.approxifer_decode_rational(p, Yt, mt, Yh), warm, iters)
+            nbytes = locate_bytes(w, m) + 4 * w.G * w.K * w.C
         elif op == "pair":
             adv = torch.empty((w.G, w.E), dtype=torch.int32, device=dev)
             trusted = torch.empty((w.G,), dtype=torch.int32, device=dev)
@@ -431,7 +438,7 @@ def main():
     ap_.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap_.add_argument("--no-cpu", action="store_true", help="skip timing the CPU checker")
     ap_.add_argument("--groups", type=int, default=None, help="override the number of groups (profiling only)")
-    ap_.add_argument("--case", default=None, choices=["decode3", "decode4", "locate5", "locateh5", "decode5", "pair5", "decode2", "encode3"],
+    ap_.add_argument("--case", default=None, choices=["decode3", "decode4", "locate5", "locateh5", "rational5", "decode5", "pair5", "decode2", "encode3"],
                      help="time one kernel of another configuration alone (tuning / profiling) and print a short JSON line")
     ap_.add_argument("--dec-config", default=None, help="stages,ctas_per_sm,disable,cols,split for the wide decoder (tuning)")
     args = ap_.parse_args()

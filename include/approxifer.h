@@ -146,6 +146,29 @@ int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C,
                       void* cuda_stream);
 
 /*
+ * Rational decoding (Algorithm 3, Appendix A: "BW-type rational interpolation in presence of errors").
+ * For every group and class the polynomials P, Q of degree < K+E with
+ *     P(beta_i) = Yt[g][i][c] * Q(beta_i),   i in the mask,   Q_0 = 1
+ * are found by least squares exactly as in approxifer_locate, and instead of locating anything the rational
+ * function itself is returned at the query nodes:
+ *     Yhat[g][j][c] = P(alpha_j) / Q(alpha_j).
+ * By the theorem that follows Algorithm 3 this equals the underlying rational function when at most E of the
+ * available predictions are wrong and at least 2(K+E) are available -- for a model that is linear in its input
+ * it returns the model's own predictions, not Berrut's approximation of them.  The paper warns that the division
+ * is numerically fragile (it amplifies the fp32 rounding of the inputs by up to ~1e5 at K+E = 10) and uses
+ * Algorithm 2 + Berrut decoding instead; this entry point is the alternative, for callers who want it.
+ *   Yt, mask   as for approxifer_locate            Yhat  out, [G][K][C]
+ *   status     out, [G] uint32 or NULL: ST_LOCATE_UNDERDETERMINED (fewer than 2(K+E) workers present; the
+ *              group's output is zero-filled), ST_NONFINITE (some output was not finite: a root of Q at alpha_j)
+ * Requires E >= 0, 2 <= K+E <= 10 and 2(K+E) <= W (APPROXIFER_E_PARAM otherwise).  The solve runs in fp64.
+ */
+int approxifer_decode_rational(const approxifer_params* params, int64_t G, int64_t C,
+                               const float* Yt, int64_t yt_gstride, int64_t yt_rstride,
+                               const uint32_t* mask,
+                               float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                               uint32_t* status, void* cuda_stream);
+
+/*
  * The decoder's two steps in one call (Section 3, "ApproxIFER Decoding", steps 1 and 2): locate the E
  * Byzantine workers of every group (Algorithm 2), then decode from the workers that are present and were
  * not located.  Equivalent to approxifer_locate followed by approxifer_decode with `trusted_mask` as the

@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     ApproxiferError,
     approxifer_debug_weights,
     approxifer_decode,
+    approxifer_decode_rational,
     approxifer_encode,
     approxifer_encode_host,
     approxifer_encode_host_static,

@@ -29,6 +29,7 @@ EXPORTS = (
     "approxifer_decode",
     "approxifer_locate",
     "approxifer_locate_decode",
+    "approxifer_decode_rational",
     "approxifer_debug_weights",
     "approxifer_strerror",
     "approxifer_version",
@@ -87,6 +88,9 @@ def load() -> ctypes.CDLL:
     lib.approxifer_locate_decode.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
                                              c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.approxifer_locate_decode.restype = c_int
+    lib.approxifer_decode_rational.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p,
+                                               c_void_p, c_int64, c_int64, c_void_p, c_void_p]
+    lib.approxifer_decode_rational.restype = c_int
     lib.approxifer_debug_weights.argtypes = [pp, c_uint32, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.approxifer_debug_weights.restype = c_int
     lib.approxifer_strerror.argtypes = [c_int]
@@ -218,6 +222,21 @@ def approxifer_locate(params: approxifer_params, Yt: torch.Tensor, mask: torch.T
     if rc != OK:
         raise ApproxiferError(rc, "approxifer_locate")
     return adv, trusted_mask
+
+
+def approxifer_decode_rational(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, Yhat: Optional[torch.Tensor] = None,
+                               status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Algorithm 3: Yhat[g][j][c] = P(alpha_j) / Q(alpha_j) with P, Q from the least-squares system of the locator."""
+    G, W, C = Yt.shape
+    if Yhat is None:
+        Yhat = torch.empty((G, params.K, C), device=Yt.device, dtype=torch.float32)
+    yp, yg, yr = _payload(Yt, params.W, "Yt")
+    op, og, orr = _payload(Yhat, params.K, "Yhat")
+    rc = load().approxifer_decode_rational(ctypes.byref(params), G, C, yp, yg, yr, _vec(mask, torch.int32, G, "mask"),
+                                           op, og, orr, _vec(status, torch.int32, G, "status"), _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_decode_rational")
+    return Yhat
 
 
 def approxifer_locate_decode(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, Yhat: Optional[torch.Tensor] = None,

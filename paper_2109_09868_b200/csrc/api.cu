@@ -82,6 +82,24 @@ int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C, con
   return from_cuda(launch_locate(a, static_cast<cudaStream_t>(cuda_stream)));
 }
 
+int approxifer_decode_rational(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
+                               int64_t yt_rstride, const uint32_t* mask, float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                               uint32_t* status, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if (params->E < 0) return APPROXIFER_E_RANGE;
+  const int m = params->K + params->E;
+  if (m < 2 || m > kLocateRowsMaxM || 2 * m > params->W) return APPROXIFER_E_PARAM;
+  if ((rc = check_layout(G, C, yt_rstride))) return rc;
+  if ((rc = check_layout(G, C, yh_rstride))) return rc;
+  if (yt_gstride < 0 || yh_gstride < 0) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (Yt == nullptr || mask == nullptr || Yhat == nullptr) return APPROXIFER_E_NULL;
+  LocateArgs a{Yt, mask, nullptr, nullptr, status, yt_gstride, yt_rstride, G, C, params->K, params->W, params->E, 0u,
+               Yhat, yh_gstride, yh_rstride};
+  return from_cuda(launch_locate(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
 int approxifer_locate_decode(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
                              int64_t yt_rstride, const uint32_t* mask, int32_t* adv, uint32_t* trusted_mask, float* Yhat,
                              int64_t yh_gstride, int64_t yh_rstride, int32_t* n_used, uint32_t* locate_status,

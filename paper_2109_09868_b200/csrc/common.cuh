@@ -47,6 +47,9 @@ struct LocateArgs {
   int64_t G, C;
   int32_t K, W, E;
   uint32_t flags;
+  // Algorithm 3 (rational decoding) only: where r(alpha_j) goes; NULL for the locator proper
+  float* Yh = nullptr;
+  int64_t o_gs = 0, o_rs = 0;
 };
 
 // Each returns a cudaError_t from the launch (cudaSuccess if nothing to do).

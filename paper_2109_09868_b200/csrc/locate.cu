@@ -270,10 +270,11 @@ void locate_config(int force_warp_kernel) { g_force_warp_kernel = force_warp_ker
 
 cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
-  const LocateTables& tab = locate_tables(a.W);
+  const LocateTables& tab = locate_tables(a.K, a.W);
   const int m = a.K + a.E;
-  // (the homogeneous form exists in the thread-per-class kernel only; the entry point has checked K+E)
-  if (m <= kLocateRowsMaxM && (!g_force_warp_kernel || (a.flags & kFlagLocateHomogeneous))) return launch_locate_rows(a, tab, stream);
+  // (the homogeneous form and Algorithm 3 exist in the thread-per-class kernel only; the entry points have checked K+E)
+  if (m <= kLocateRowsMaxM && (!g_force_warp_kernel || (a.flags & kFlagLocateHomogeneous) || a.Yh != nullptr))
+    return launch_locate_rows(a, tab, stream);
   if (a.W <= 8) return dispatch_m<8>(m, a, tab, stream);
   if (a.W <= 16) return dispatch_m<16>(m, a, tab, stream);
   if (a.W <= 24) return dispatch_m<24>(m, a, tab, stream);

@@ -40,6 +40,21 @@ struct GroupSmem {
   int pad;
 };
 
+// Bytes of the per-CTA scratch: the threads' predictions, or (during set-up) the warps' reflectors and the
+// transposed full-set basis, whichever is larger.
+template <int NMAX, int M>
+__host__ __device__ constexpr size_t scratch_bytes() {
+  const size_t y_bytes = (size_t)NMAX * kRowsThreads * sizeof(float);
+  const size_t setup_bytes = ((size_t)kRowsWarps * M + (NMAX - M)) * NMAX * sizeof(double);
+  return y_bytes > setup_bytes ? y_bytes : setup_bytes;
+}
+
+// The k-th of M ranks spread evenly over 0 .. n-1 (first and last included).
+template <int M>
+__host__ __device__ __forceinline__ int spread_rank(int k, int n) {
+  return (k * (n - 1)) / (M - 1);
+}
+
 template <int NMAX, int M, int K0 = 0>
 __device__ __forceinline__ void rows_pblock_factor(double (&col)[NMAX], int lane, double (*refl)[NMAX]) {
   if constexpr (K0 < M) {
@@ -210,9 +225,13 @@ __device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double 
 }
 
 
-// HOMOG: Algorithm 1's homogeneous system (Q_0 free) solved in the least-squares sense with |Q| = 1, instead of
-// Algorithm 2's normalisation Q_0 = 1; everything else (basis, rows, selection, vote) is shared.
-template <int NMAX, int M, bool HOMOG>
+// MODE 0: Algorithm 2 (Q_0 = 1).  MODE 1: Algorithm 1's homogeneous system (Q_0 free) solved in the least-squares
+// sense with |Q| = 1; basis, rows, selection and vote are shared.  MODE 2: Algorithm 3 -- the same per-class
+// solve as mode 0, then no selection and no vote: P is recovered and r = P/Q is evaluated at the K nodes alpha_j
+// (a decoder that absorbs up to E wrong predictions instead of locating them).
+constexpr int kModeLocate = 0, kModeHomogeneous = 1, kModeRational = 2;
+
+template <int NMAX, int M, int MODE>
 __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __grid_constant__ LocateArgs a,
                                                                       const __grid_constant__ LocateTables tab,
                                                                       const __grid_constant__ LocateBasis basis,
@@ -227,9 +246,13 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
   unsigned char* scratch = smem_raw + (size_t)gpb * sizeof(SM);
   float* ysm = reinterpret_cast<float*>(scratch) + threadIdx.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr bool HOMOG = MODE == kModeHomogeneous;
   const int E = a.E;
   const int64_t g_first = (int64_t)blockIdx.x * gpb;
   const int ng = (int)min((int64_t)gpb, a.G - g_first);
+
+  // (Algorithm 3 only) per group, behind the scratch: the K x M table that carries P from M nodes to the alpha_j
+  double* lgs = reinterpret_cast<double*>(scratch + scratch_bytes<NMAX, M>());
 
   // ---- set-up, one warp per group ------------------------------------------------------------------
   {
@@ -242,6 +265,27 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
     for (int s = warp; s < ng; s += kRowsWarps) {
       rows_setup_group<NMAX, M>(groups[s], refl, nft, a, tab, g_first + s, lane);
       __syncwarp();  // the scratch is reused by this warp's next group
+      if constexpr (MODE == kModeRational) {
+        // P has degree < M, so its values on M of the available nodes (spread over the whole range) fix it:
+        // lg[j][k] = Lagrange basis of those nodes at alpha_j, lane = j
+        const SM& sm = groups[s];
+        if (sm.n >= 0 && lane < a.K) {
+          double* lg = lgs + (size_t)s * M * M + lane * M;
+          const double z = tab.alpha[lane];
+#pragma unroll 1
+          for (int k = 0; k < M; ++k) {
+            const double xk = sm.xs[spread_rank<M>(k, sm.n)];
+            double num = 1.0, den = 1.0;
+            for (int l = 0; l < M; ++l) {
+              if (l == k) continue;
+              const double xl = sm.xs[spread_rank<M>(l, sm.n)];
+              num *= z - xl;
+              den *= xk - xl;
+            }
+            lg[k] = num / den;
+          }
+        }
+      }
     }
   }
   __syncthreads();
@@ -253,7 +297,11 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
     const int64_t c = t - (int64_t)s * a.C;
     SM& sm = groups[s];
     const int n = sm.n;
-    if (n < 0) continue;
+    if (n < 0) {
+      if constexpr (MODE == kModeRational)  // nothing can be solved: the group's output is zero-filled
+        for (int j = 0; j < a.K; ++j) a.Yh[(g_first + s) * a.o_gs + j * a.o_rs + c] = 0.f;
+      continue;
+    }
     const float* Yc = a.Yt + (g_first + s) * a.y_gs + c;
 
 #pragma unroll
@@ -381,6 +429,56 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
       }
     }
 
+    if constexpr (MODE == kModeRational) {
+      // Algorithm 3, Step 2.  For this Q the best P is the least-squares polynomial through (b_i, y_i Q(b_i)):
+      // on the nodes, P = t - N (N^T t) with t_i = y_i a_i.  Its values on M spread nodes carry it to alpha_j.
+      double z[NMAX - M];
+#pragma unroll
+      for (int r = 0; r < NMAX - M; ++r) z[r] = 0.0;
+#pragma unroll 2
+      for (int i = 0; i < NMAX; ++i) {
+        const double b = sm.xs[i];
+        double h = q[NC - 1];
+#pragma unroll
+        for (int k = NC - 2; k >= 0; --k) h = fma(h, b, q[k]);
+        const double ti = (i < n) ? fma(h, b, 1.0) * (double)ysm[i * kRowsThreads] : 0.0;
+#pragma unroll
+        for (int r = 0; r < NMAX - M; ++r)
+          if (r < rows) z[r] = fma(sm.nt[r][i], ti, z[r]);  // N has n-M columns; the rest of nt is not meaningful
+      }
+      double pk[M];
+#pragma unroll
+      for (int k = 0; k < M; ++k) {
+        const int i = spread_rank<M>(k, n);
+        const double b = sm.xs[i];
+        double h = q[NC - 1];
+#pragma unroll
+        for (int kk = NC - 2; kk >= 0; --kk) h = fma(h, b, q[kk]);
+        double v = fma(h, b, 1.0) * (double)ysm[i * kRowsThreads];
+#pragma unroll
+        for (int r = 0; r < NMAX - M; ++r)
+          if (r < rows) v = fma(-sm.nt[r][i], z[r], v);
+        pk[k] = v;
+      }
+      const double* lg = lgs + (size_t)s * M * M;
+      float* out = a.Yh + (g_first + s) * a.o_gs + (t - (int64_t)s * a.C);
+      bool nonfin = false;
+      for (int j = 0; j < a.K; ++j) {
+        double pv = 0.0;
+#pragma unroll
+        for (int k = 0; k < M; ++k) pv = fma(lg[j * M + k], pk[k], pv);
+        const double zj = tab.alpha[j];
+        double h = q[NC - 1];
+#pragma unroll
+        for (int kk = NC - 2; kk >= 0; --kk) h = fma(h, zj, q[kk]);
+        const float o = (float)(pv / fma(h, zj, 1.0));
+        nonfin |= !isfinite(o);
+        out[j * a.o_rs] = o;
+      }
+      if (nonfin) atomicOr(&sm.status, kStNonfinite);
+      continue;
+    }
+
     // a_i = Q(b_i) = 1 + sum_k q_k b_i^(k+1); the E smallest |a_i| (ties to the lower worker) get a vote
     double mag[NMAX];
     bool nonfinite = false;
@@ -414,6 +512,10 @@ __global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __gr
   }
   __syncthreads();
 
+  if constexpr (MODE == kModeRational) {
+    if (a.status != nullptr && tid < ng) a.status[g_first + tid] = groups[tid].status;
+    return;
+  }
   // ---- the E most voted workers of each group, ties to the lower index; lane = rank ----------------
   for (int s = warp; s < ng; s += kRowsWarps) {
     const SM& sm = groups[s];
@@ -455,11 +557,10 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
   // as many groups per CTA as give every thread a class, within the shared-memory budget of two CTAs per SM
   int64_t gpb = a.C >= kRowsThreads ? 1 : kRowsThreads / a.C;
   if (gpb > kMaxGroupsPerCta) gpb = kMaxGroupsPerCta;
-  const size_t per_group = sizeof(GroupSmem<NMAX, M>);
-  size_t y_bytes = (size_t)NMAX * kRowsThreads * sizeof(float);  // per-thread predictions ...
-  // ... aliased with the set-up scratch: the warps' reflectors and the transposed full-set basis
-  const size_t refl_bytes = ((size_t)kRowsWarps * M + (NMAX - M)) * NMAX * sizeof(double);
-  if (refl_bytes > y_bytes) y_bytes = refl_bytes;
+  // per group: its block, and for Algorithm 3 the M x M table that carries P to the alpha nodes
+  const size_t per_group = sizeof(GroupSmem<NMAX, M>) + (a.Yh != nullptr ? (size_t)M * M * sizeof(double) : 0);
+  // per-thread predictions, aliased with the set-up scratch (the warps' reflectors and the transposed full-set basis)
+  const size_t y_bytes = scratch_bytes<NMAX, M>();
   while (gpb > 1 && gpb * per_group + y_bytes > 74 * 1024) --gpb;
   if (gpb > a.G) gpb = a.G;
   const size_t smem = (size_t)gpb * per_group + y_bytes;
@@ -474,8 +575,9 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
     count_launch();
     return cudaGetLastError();
   };
-  if (a.flags & kFlagLocateHomogeneous) return run(locate_rows_kernel<NMAX, M, true>);
-  return run(locate_rows_kernel<NMAX, M, false>);
+  if (a.Yh != nullptr) return run(locate_rows_kernel<NMAX, M, kModeRational>);
+  if (a.flags & kFlagLocateHomogeneous) return run(locate_rows_kernel<NMAX, M, kModeHomogeneous>);
+  return run(locate_rows_kernel<NMAX, M, kModeLocate>);
 }
 
 template <int NMAX, int M = 2>

@@ -70,10 +70,12 @@ void build_decode_tables(int K, int W, DecodeTables* t) {
     }
 }
 
-void build_locate_tables(int W, LocateTables* t) {
+void build_locate_tables(int K, int W, LocateTables* t) {
   std::memset(t, 0, sizeof(*t));
   // beta_i = cos(pi i/(W-1)) = sin(pi (1/2 - i/(W-1)))
   for (int i = 0; i < W; ++i) t->beta[i] = (double)sinpi_ratio((long long)(W - 1) - 2 * i, 2LL * (W - 1));
+  // alpha_j = cos(pi (2j+1)/(2K)) = sin(pi (K - 2j - 1)/(2K))
+  for (int j = 0; j < K; ++j) t->alpha[j] = (double)sinpi_ratio((long long)K - 2 * j - 1, 2LL * K);
 }
 
 void build_locate_basis(int W, int M, LocateBasis* t) {
@@ -145,10 +147,10 @@ const DecodeTables& decode_tables(int K, int W) {
   return cached(cache, mu, K * 64 + W, [&](DecodeTables* t) { build_decode_tables(K, W, t); });
 }
 
-const LocateTables& locate_tables(int W) {
+const LocateTables& locate_tables(int K, int W) {
   static std::map<int, std::unique_ptr<LocateTables>> cache;
   static std::mutex mu;
-  return cached(cache, mu, W, [&](LocateTables* t) { build_locate_tables(W, t); });
+  return cached(cache, mu, K * 64 + W, [&](LocateTables* t) { build_locate_tables(K, W, t); });
 }
 
 const LocateBasis& locate_basis(int W, int M) {

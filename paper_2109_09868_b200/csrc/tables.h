@@ -24,9 +24,10 @@ struct EncodeTables {
   float w[kMaxW * kMaxK];
 };
 
-// beta_i in double for the locator.
+// beta_i (and alpha_j, for Algorithm 3) in double for the locator.
 struct LocateTables {
   double beta[kMaxW];
+  double alpha[kMaxK];
 };
 
 // Orthonormal basis Nf of the orthogonal complement of {polynomials of degree < M} on the FULL node set
@@ -47,7 +48,7 @@ long double node_gap(int K, int W, int j, int i);
 
 void build_encode_tables(int K, int W, EncodeTables* t);
 void build_decode_tables(int K, int W, DecodeTables* t);
-void build_locate_tables(int W, LocateTables* t);
+void build_locate_tables(int K, int W, LocateTables* t);
 void build_locate_basis(int W, int M, LocateBasis* t);
 
 // The tables depend on (K, W) only and cost 10-200 us of host time to build, so each is built once per
@@ -55,7 +56,7 @@ void build_locate_basis(int W, int M, LocateBasis* t);
 // for the life of the process.
 const EncodeTables& encode_tables(int K, int W);
 const DecodeTables& decode_tables(int K, int W);
-const LocateTables& locate_tables(int W);
+const LocateTables& locate_tables(int K, int W);
 const LocateBasis& locate_basis(int W, int M);
 
 }  // namespace approxifer
