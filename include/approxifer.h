@@ -5,7 +5,8 @@
  * The library implements the data-parallel hot path of ApproxIFER
  * (arXiv 2109.09868, Section 3): the Berrut rational-interpolation encoder,
  * the straggler-masked Berrut decoder and the Byzantine-worker locator
- * (Algorithm 2), over G independent groups at a time.
+ * (Algorithm 2; Algorithm 1's homogeneous system and Algorithm 3's rational
+ * function as alternatives), over G independent groups at a time.
  *
  * Notation.  K = queries per group (j = 0..K-1).  W = number of workers =
  * number of coded queries (i = 0..W-1); the paper counts workers 0..N, so

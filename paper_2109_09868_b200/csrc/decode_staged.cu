@@ -9,13 +9,13 @@
 // reduced from shared memory.  Nothing waits on a register-staged load and the
 // register file holds only the accumulators.
 //
-// A work item is (group, tile of COLS 16-byte columns).  2*COLS compute threads
-// work on it: thread = (half, column); half h forms the queries
-// j = h*KT .. h*KT+KT-1 (KT = ceil(K/SPLIT)), so two warps share each column's
-// payload but every thread keeps only KT accumulators per payload element,
-// which doubles the warps per byte of ring.  The FMAs are packed
-// (fma.rn.f32x2: the weights of two adjacent queries times one payload
-// element, each half an ordinary round-to-nearest fp32 FMA).  One more warp is
+// A work item is (group, tile of COLS 16-byte columns).  SPLIT*COLS compute threads work on it:
+// thread = (thread group h, column); group h forms the queries j = h*KT .. h*KT+KT-1 (KT = ceil(K/SPLIT)).
+// With SPLIT = 1 (the default where it fits: K <= 16, COLS = 256, one CTA per SM) every payload word is read
+// from shared memory once and a thread keeps all K accumulators per payload element; with SPLIT = 2 or 4 the
+// thread groups share each column's payload, every thread keeps only KT accumulators, and there are more warps
+// per byte of ring (two CTAs per SM).  The FMAs are packed (fma.rn.f32x2: the weights of two adjacent
+// queries times one payload element, each half an ordinary round-to-nearest fp32 FMA).  One more warp is
 // the producer: for each item it waits for a free ring slot, writes the item's
 // signed weights (by rank) and K reciprocal denominators into the slot, and
 // starts the copies of the present rows; slots are handed over and back

@@ -1,18 +1,21 @@
-// ApproxIFER Byzantine-worker locator (Algorithm 2), thread-per-class variant for K+E <= 10.
+// ApproxIFER Byzantine-worker locator (Algorithm 2), thread-per-class variant for K+E <= 10; also Algorithm 1's
+// homogeneous system and Algorithm 3's rational function as alternative last steps (see the kernel's MODE).
 //
 // Same mathematics as locate_kernel (locate.cu): the P-part of the per-class least-squares problem is
 // eliminated with an orthonormal basis N of the complement of {polynomials of degree < M} on the available
 // nodes (M = K+E), which depends on the mask only, and the Q-part solves the (n-M) x (M-1) problem
 //     B q = -b0,   B[r][l] = sum_i N[i][r] y_i b_i^l (l = 1..M-1),   b0[r] = sum_i N[i][r] y_i.
-// Different parallelisation: after one warp per group has produced N (Householder reflectors of the
-// Vandermonde block applied to unit vectors, lane = column), every (group, class) pair gets ONE THREAD.
+// Different parallelisation: after one warp per group has produced N (from the basis of the full node set by a
+// few small reflectors when few workers are missing, else by Householder reflectors of the group's own
+// Vandermonde block applied to unit vectors), every (group, class) pair gets ONE THREAD.
 // The thread generates the rows of [B | -b0] one at a time from N (shared memory, shared by the group's
-// threads) and its own 22-odd predictions (registers) and folds each row into an upper-triangular factor
-// with Givens rotations.  The factor (at most 45 + 9 doubles) lives in registers with static indices; the
-// rows are never stored.  No lane waits for another lane: there is no serial single-lane section, and all
-// 32 lanes of a warp work on different problems.  The thread then evaluates a_r = Q(b_r) for every
-// available worker, picks the E smallest |a_r| (ties to the lower worker) and votes with shared-memory
-// atomics; a warp per group elects the E most voted workers.  Everything runs in fp64.
+// threads) and its own 22-odd predictions (shared memory, one column per thread) and folds each row into a
+// square-root-free triangular factor (Gentleman's form of the Givens row update).  The factor (at most
+// 45 + 9 doubles) lives in registers with static indices; the rows are never stored.  No lane waits for
+// another lane: there is no serial single-lane section, and all 32 lanes of a warp work on different
+// problems.  The thread then evaluates a_r = Q(b_r) for every available worker, picks the E smallest |a_r|
+// (ties to the lower worker) and votes with shared-memory atomics; a warp per group elects the E most voted
+// workers.  Everything runs in fp64.
 #include "common.cuh"
 #include "locate_common.cuh"
 
