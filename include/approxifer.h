@@ -274,7 +274,7 @@ int approxifer_debug_decode_config(int stages, int ctas_per_sm, int disable, int
 
 /*
  * Test hook for the locator: force_warp_kernel != 0 routes every locate through the
- * warp-per-group kernel, which otherwise serves only K+E > 10 (smaller K+E use the
+ * warp-per-group kernel, which otherwise serves only K+E > 15 (smaller K+E use the
  * thread-per-class kernel).  Both follow Algorithm 2 and return the same sets.
  * Process-wide, not thread-safe.
  */

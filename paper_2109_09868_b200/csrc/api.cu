@@ -73,7 +73,7 @@ int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C, con
   if (rc) return rc;
   if (params->E < 0) return APPROXIFER_E_RANGE;
   if (params->E < 1 || 2 * (params->K + params->E) > params->W) return APPROXIFER_E_PARAM;
-  if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateRowsMaxM) return APPROXIFER_E_PARAM;
+  if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateAltMaxM) return APPROXIFER_E_PARAM;
   if ((rc = check_layout(G, C, yt_rstride))) return rc;
   if (yt_gstride < 0) return APPROXIFER_E_RANGE;
   if (G == 0) return APPROXIFER_OK;
@@ -89,7 +89,7 @@ int approxifer_decode_rational(const approxifer_params* params, int64_t G, int64
   if (rc) return rc;
   if (params->E < 0) return APPROXIFER_E_RANGE;
   const int m = params->K + params->E;
-  if (m < 2 || m > kLocateRowsMaxM || 2 * m > params->W) return APPROXIFER_E_PARAM;
+  if (m < 2 || m > kLocateAltMaxM || 2 * m > params->W) return APPROXIFER_E_PARAM;
   if ((rc = check_layout(G, C, yt_rstride))) return rc;
   if ((rc = check_layout(G, C, yh_rstride))) return rc;
   if (yt_gstride < 0 || yh_gstride < 0) return APPROXIFER_E_RANGE;

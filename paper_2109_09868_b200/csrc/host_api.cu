@@ -154,7 +154,7 @@ int approxifer_locate_host(const approxifer_params* params, int64_t G, int64_t C
     return APPROXIFER_E_RANGE;
   if (params->E < 1 || 2 * (params->K + params->E) > params->W) return APPROXIFER_E_PARAM;
   if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS)) return APPROXIFER_E_PARAM;
-  if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateRowsMaxM) return APPROXIFER_E_PARAM;
+  if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateAltMaxM) return APPROXIFER_E_PARAM;
   if (G < 0 || C < 1 || C > (int64_t(1) << 31)) return APPROXIFER_E_RANGE;
   if (G == 0) return APPROXIFER_OK;
   if (hYt == nullptr || hmask == nullptr || hadv == nullptr || htrusted == nullptr || workspace == nullptr ||

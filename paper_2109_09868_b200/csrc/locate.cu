@@ -273,7 +273,8 @@ cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream) {
   const LocateTables& tab = locate_tables(a.K, a.W);
   const int m = a.K + a.E;
   // (the homogeneous form and Algorithm 3 exist in the thread-per-class kernel only; the entry points have checked K+E)
-  if (m <= kLocateRowsMaxM && (!g_force_warp_kernel || (a.flags & kFlagLocateHomogeneous) || a.Yh != nullptr))
+  const bool alt = (a.flags & kFlagLocateHomogeneous) || a.Yh != nullptr;
+  if (alt ? m <= kLocateAltMaxM : (m <= kLocateRowsMaxM && !g_force_warp_kernel))
     return launch_locate_rows(a, tab, stream);
   if (a.W <= 8) return dispatch_m<8>(m, a, tab, stream);
   if (a.W <= 16) return dispatch_m<16>(m, a, tab, stream);

@@ -1,4 +1,4 @@
-// ApproxIFER Byzantine-worker locator (Algorithm 2), thread-per-class variant for K+E <= 10; also Algorithm 1's
+// ApproxIFER Byzantine-worker locator (Algorithm 2), thread-per-class variant for K+E <= 15; also (K+E <= 10) Algorithm 1's
 // homogeneous system and Algorithm 3's rational function as alternative last steps (see the kernel's MODE).
 //
 // Same mathematics as locate_kernel (locate.cu): the P-part of the per-class least-squares problem is
@@ -235,7 +235,7 @@ __device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double 
 constexpr int kModeLocate = 0, kModeHomogeneous = 1, kModeRational = 2;
 
 template <int NMAX, int M, int MODE>
-__global__ void __launch_bounds__(kRowsThreads, 3) locate_rows_kernel(const __grid_constant__ LocateArgs a,
+__global__ void __launch_bounds__(kRowsThreads, M > 10 ? 2 : 3) locate_rows_kernel(const __grid_constant__ LocateArgs a,
                                                                       const __grid_constant__ LocateTables tab,
                                                                       const __grid_constant__ LocateBasis basis,
                                                                       const int gpb) {
@@ -564,7 +564,10 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
   const size_t per_group = sizeof(GroupSmem<NMAX, M>) + (a.Yh != nullptr ? (size_t)M * M * sizeof(double) : 0);
   // per-thread predictions, aliased with the set-up scratch (the warps' reflectors and the transposed full-set basis)
   const size_t y_bytes = scratch_bytes<NMAX, M>();
-  while (gpb > 1 && gpb * per_group + y_bytes > 74 * 1024) --gpb;
+  // shared memory for three CTAs per SM (K+E <= 10: 168 registers per thread) or two (the larger factors
+  // of K+E = 11..15 take 255 registers, and from 14 on a little local memory)
+  const size_t budget = (M > 10 ? 110 : 74) * 1024;
+  while (gpb > 1 && gpb * per_group + y_bytes > budget) --gpb;
   if (gpb > a.G) gpb = a.G;
   const size_t smem = (size_t)gpb * per_group + y_bytes;
   const int64_t blocks = (a.G + gpb - 1) / gpb;
@@ -578,8 +581,10 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
     count_launch();
     return cudaGetLastError();
   };
-  if (a.Yh != nullptr) return run(locate_rows_kernel<NMAX, M, kModeRational>);
-  if (a.flags & kFlagLocateHomogeneous) return run(locate_rows_kernel<NMAX, M, kModeHomogeneous>);
+  if constexpr (M <= kLocateAltMaxM) {
+    if (a.Yh != nullptr) return run(locate_rows_kernel<NMAX, M, kModeRational>);
+    if (a.flags & kFlagLocateHomogeneous) return run(locate_rows_kernel<NMAX, M, kModeHomogeneous>);
+  }
   return run(locate_rows_kernel<NMAX, M, kModeLocate>);
 }
 

@@ -299,7 +299,7 @@ def compare_locate(K, W, E, Yt, mask, allow_fragile=False):
     return ref, adv, int((~solid).sum())
 
 
-@pytest.mark.parametrize("K,E,S,W", [(8, 2, 2, 24), (2, 1, 0, 6), (3, 2, 1, 12), (4, 1, 2, 12), (12, 2, 0, 28),
+@pytest.mark.parametrize("K,E,S,W", [(8, 2, 2, 24), (2, 1, 0, 6), (3, 2, 1, 12), (4, 1, 2, 12), (12, 2, 0, 28), (12, 1, 2, 28), (10, 3, 0, 26),
                                      (6, 3, 1, 20), (1, 1, 0, 4), (13, 3, 0, 32), (8, 2, 0, 20), (2, 1, 3, 9)])
 def test_locate_matches_oracle_and_finds_injected_errors(K, E, S, W):
     G, C = 96, 10
@@ -470,9 +470,12 @@ def test_worker_major_layouts_for_decode_and_locate():
         check_decode(K, W, Yt, ref["trusted"], out.permute(1, 0, 2))
 
 
-@pytest.mark.parametrize("K,E,S,W,C", [(8, 2, 2, 24, 10), (3, 2, 1, 12, 37), (4, 1, 2, 12, 300), (2, 1, 0, 6, 1), (7, 3, 1, 22, 10)])
+@pytest.mark.parametrize("K,E,S,W,C", [(8, 2, 2, 24, 10), (3, 2, 1, 12, 37), (4, 1, 2, 12, 300), (2, 1, 0, 6, 1), (7, 3, 1, 22, 10),
+                                       (10, 1, 0, 22, 10), (10, 2, 3, 27, 10), (12, 1, 0, 26, 10), (10, 3, 2, 28, 7), (11, 2, 6, 32, 10),
+                                       (9, 2, 1, 23, 140), (12, 2, 0, 28, 10), (12, 3, 1, 31, 10), (13, 2, 2, 32, 5)])
 def test_both_locator_kernels_return_the_same_sets(K, E, S, W, C):
-    """K+E <= 10 normally takes the thread-per-class kernel; the warp-per-group kernel must agree with it
+    """K+E <= 15 normally takes the thread-per-class kernel (two CTAs per SM for K+E = 11..15, whose factor needs
+    255 registers and, from 14 on, some local memory); the warp-per-group kernel must agree with it
     (and with the oracle) on the same inputs, including groups with too few workers."""
     G = 150
     Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=K + 7 * E + C)
