@@ -56,7 +56,7 @@ extern "C" {
 #define APPROXIFER_OK 0
 #define APPROXIFER_E_NULL (-1)  /* a required pointer is NULL */
 #define APPROXIFER_E_RANGE (-2) /* K not in 1..32, W not in 2..32, E < 0, G < 0, D < 1, D > 2^31, stride < row length */
-#define APPROXIFER_E_PARAM (-3) /* locate: E < 1, 2(K+E) > W, or the homogeneous form with K+E > 10; unknown flag bits */
+#define APPROXIFER_E_PARAM (-3) /* locate: E < 1, 2(K+E) > W, or the homogeneous form with K+E > 13; unknown flag bits */
 #define APPROXIFER_E_CUDA (-4)  /* the CUDA runtime reported an error at launch */
 #define APPROXIFER_E_WORKSPACE (-5) /* host-buffer entry points: the device workspace cannot hold one group */
 #define APPROXIFER_E_TOO_LARGE (-6) /* approxifer_encode_host_static: the batch does not fit the built-in staging area */
@@ -138,7 +138,7 @@ int approxifer_decode(const approxifer_params* params, int64_t G, int64_t C,
  * all P and over Q with sum_k Q_k^2 = 1 (the smallest singular direction).
  * Selection, vote, outputs and status bits are the same.  This form has no
  * special case at a node equal to 0 (odd W), where Q_0 = 1 pins a_i to 1.
- * Available for K+E <= 10; APPROXIFER_E_PARAM otherwise.
+ * Available for K+E <= 13; APPROXIFER_E_PARAM otherwise.
  */
 int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C,
                       const float* Yt, int64_t yt_gstride, int64_t yt_rstride,
@@ -161,7 +161,7 @@ int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C,
  *   Yt, mask   as for approxifer_locate            Yhat  out, [G][K][C]
  *   status     out, [G] uint32 or NULL: ST_LOCATE_UNDERDETERMINED (fewer than 2(K+E) workers present; the
  *              group's output is zero-filled), ST_NONFINITE (some output was not finite: a root of Q at alpha_j)
- * Requires E >= 0, 2 <= K+E <= 10 and 2(K+E) <= W (APPROXIFER_E_PARAM otherwise).  The solve runs in fp64.
+ * Requires E >= 0, 2 <= K+E <= 13 and 2(K+E) <= W (APPROXIFER_E_PARAM otherwise).  The solve runs in fp64.
  */
 int approxifer_decode_rational(const approxifer_params* params, int64_t G, int64_t C,
                                const float* Yt, int64_t yt_gstride, int64_t yt_rstride,

@@ -73,7 +73,7 @@ void decode_small_config(int disable);
 // Thread-per-class locator for K+E <= kLocateRowsMaxM (locate_rows.cu); the warp-per-group kernel covers the rest.
 constexpr int kLocateRowsMaxM = 15;
 // ... and its alternative last steps (Algorithm 1's homogeneous system, Algorithm 3) for K+E <= kLocateAltMaxM
-constexpr int kLocateAltMaxM = 10;
+constexpr int kLocateAltMaxM = 13;
 cudaError_t launch_locate_rows(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream);
 void locate_config(int force_warp_kernel);
 

@@ -1,4 +1,4 @@
-// ApproxIFER Byzantine-worker locator (Algorithm 2), thread-per-class variant for K+E <= 15; also (K+E <= 10) Algorithm 1's
+// ApproxIFER Byzantine-worker locator (Algorithm 2), thread-per-class variant for K+E <= 15; also (K+E <= 13) Algorithm 1's
 // homogeneous system and Algorithm 3's rational function as alternative last steps (see the kernel's MODE).
 //
 // Same mathematics as locate_kernel (locate.cu): the P-part of the per-class least-squares problem is

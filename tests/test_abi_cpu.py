@@ -74,8 +74,8 @@ def test_decode_and_locate_argument_errors():
         assert rc == want, (K, W, E)
     q = ap.make_params(8, 24, 2)
     assert lib.approxifer_locate(ctypes.byref(q), 1, 10, 1, 240, 10, 1, None, 1, None, None) == binding.E_NULL
-    # the homogeneous form of the locator exists for K+E <= 10
-    for (K, W, E, want) in [(8, 24, 2, binding.OK), (9, 32, 2, binding.E_PARAM), (12, 32, 2, binding.E_PARAM)]:
+    # the homogeneous form of the locator exists for K+E <= 13
+    for (K, W, E, want) in [(8, 24, 2, binding.OK), (9, 32, 2, binding.OK), (12, 32, 1, binding.OK), (12, 32, 2, binding.E_PARAM)]:
         q = ap.make_params(K, W, E, binding.LOCATE_HOMOGENEOUS)
         assert lib.approxifer_locate(ctypes.byref(q), 0, 10, None, W * 10, 10, None, None, None, None, None) == want
 

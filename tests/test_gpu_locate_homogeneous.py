@@ -71,7 +71,7 @@ def compare(K, W, E, Yt, mask, allow_fragile=False):
 
 @pytest.mark.parametrize("K,E,S,W", [(8, 2, 2, 24), (2, 1, 0, 6), (3, 2, 1, 12), (4, 1, 2, 12), (6, 3, 1, 20),
                                      (1, 1, 0, 4), (7, 3, 0, 32), (8, 2, 0, 20), (2, 1, 3, 9), (3, 2, 1, 11),
-                                     (5, 1, 9, 21)])
+                                     (5, 1, 9, 21), (10, 1, 0, 22), (12, 1, 0, 26), (10, 3, 1, 27)])
 def test_homogeneous_locator_matches_oracle_and_finds_injected_errors(K, E, S, W):
     G, C = 96, 10
     Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=K * 37 + E)
