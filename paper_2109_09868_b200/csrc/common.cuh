@@ -70,7 +70,7 @@ bool decode_small_eligible(const DecodeArgs& a);
 cudaError_t launch_decode_small(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream);
 void decode_small_config(int disable);
 
-// Thread-per-class locator for K+E <= kLocateRowsMaxM (locate_rows.cu); the warp-per-group kernel covers the rest.
+// Thread-per-class locator for K+E <= kLocateRowsMaxM (locate_rows_impl.cuh); the warp-per-group kernel covers the rest.
 constexpr int kLocateRowsMaxM = 15;
 // ... and its alternative last steps (Algorithm 1's homogeneous system, Algorithm 3) for K+E <= kLocateAltMaxM
 constexpr int kLocateAltMaxM = 13;
