@@ -209,7 +209,7 @@ def physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
-def time_launches(fn, warmup=3, iters=10):
+def time_launches(fn, warmup=3, iters=10, all_times=None):
     """Per-launch device time (ms) of fn() on the current stream: median and min."""
     for _ in range(warmup):
         fn()
@@ -221,6 +221,8 @@ def time_launches(fn, warmup=3, iters=10):
         b.record()
     torch.cuda.synchronize()
     ms = [a.elapsed_time(b) for a, b in evs]
+    if all_times is not None:
+        all_times.extend(ms)
     return statistics.median(ms), min(ms)
 
 
@@ -278,9 +280,16 @@ def other_workloads(ap, dev, peak):
     m4 = wl.masks(w4g)
     mt = ap.mask_tensor(m4, dev)
     Yh = torch.empty((G4, w4.K, w4.C), device=dev)
-    med, mn = time_launches(lambda: ap.approxifer_decode(p4, Yt, mt, Yh), 3, 10)
-    entry("configs[3] decode K=16 W=24 C=1000, 16-24 present", decode_bytes(w4g, m4), med, mn, G4,
-          {"note": "all 262144 groups" if G4 == w4.G else "G reduced to fit free device memory"})
+    # 40 launches back to back: the first ones run at boost clocks, then the board's power cap lowers the SM clock
+    # and the launch time settles; the headline figure of this entry is the median of all 40, both regimes are given
+    times4 = []
+    med, mn = time_launches(lambda: ap.approxifer_decode(p4, Yt, mt, Yh), 3, 40, times4)
+    nb4 = decode_bytes(w4g, m4)
+    entry("configs[3] decode K=16 W=24 C=1000, 16-24 present", nb4, med, mn, G4,
+          {"note": "all 262144 groups" if G4 == w4.G else "G reduced to fit free device memory",
+           "launches": len(times4),
+           "first5_ms": statistics.median(times4[:5]), "first5_GB_per_s": nb4 / statistics.median(times4[:5]) / 1e6,
+           "last20_ms": statistics.median(times4[-20:]), "last20_GB_per_s": nb4 / statistics.median(times4[-20:]) / 1e6})
     del Yt, Yh
     torch.cuda.empty_cache()
 
