@@ -39,9 +39,9 @@ HEADLINE_CFG = 2
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic of encode_kernel<8, float4> per group of the headline workload, from the ncu capture of a
-# 4096-group launch: (402.663 MB read + 546.9 MB written) / 4096.  Traffic is proportional to the number
+# 4096-group launch: (402.664 MB read + 548.5 MB written) / 4096.  Traffic is proportional to the number
 # of groups (every row is touched once); the written part misses the dirty lines still in L2 at kernel end.
-ENCODE_TRAFFIC_PER_GROUP = (402.663e6 + 546.9e6) / 4096
+ENCODE_TRAFFIC_PER_GROUP = (402.664e6 + 548.5e6) / 4096
 
 
 # ----------------------------------------------------------------- byte counts

@@ -12,6 +12,7 @@ namespace approxifer {
 namespace {
 
 constexpr int kEncodeThreads = 256;
+constexpr int kEncodeWideThreads = 768;
 
 template <typename V>
 struct VecOps;
@@ -33,12 +34,12 @@ struct VecOps<float> {
 // One work item = (group g, column v) with v counting V-wide columns of the
 // payload; items are numbered g*Dv + v and dealt to threads in order, so a
 // warp reads and writes 32 consecutive columns of a row.
-template <int K, typename V>
-__global__ void __launch_bounds__(kEncodeThreads) encode_kernel(const __grid_constant__ EncodeArgs a,
-                                                                const __grid_constant__ EncodeTables tab) {
+template <int K, typename V, int THREADS>
+__global__ void __launch_bounds__(THREADS) encode_kernel(const __grid_constant__ EncodeArgs a,
+                                                         const __grid_constant__ EncodeTables tab) {
   using Ops = VecOps<V>;
   const uint32_t Dv = (uint32_t)(a.D / Ops::kLanes);
-  const int64_t first = (int64_t)blockIdx.x * kEncodeThreads;  // first item of this block
+  const int64_t first = (int64_t)blockIdx.x * THREADS;  // first item of this block
   const int64_t g0 = first / Dv;
   const uint32_t t = (uint32_t)(first - g0 * Dv) + threadIdx.x;
   const uint32_t dg = t / Dv;
@@ -69,9 +70,18 @@ template <int K, typename V>
 cudaError_t launch_one(const EncodeArgs& a, const EncodeTables& tab, cudaStream_t stream) {
   const int64_t Dv = a.D / VecOps<V>::kLanes;
   const int64_t items = a.G * Dv;
-  const int64_t blocks = (items + kEncodeThreads - 1) / kEncodeThreads;
-  if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-  encode_kernel<K, V><<<(unsigned)blocks, kEncodeThreads, 0, stream>>>(a, tab);
+  // Rows that tile exactly into pieces of 768 columns (12 KB: a whole row of a 3x32x32 query) get CTAs of that
+  // size: each CTA then reads and writes whole contiguous pieces of K and W rows, which HBM serves slightly
+  // better (+0.8 % on workload 2) than the 4 KB pieces of 256-thread CTAs.
+  if (VecOps<V>::kLanes == 4 && Dv % kEncodeWideThreads == 0) {
+    const int64_t blocks = items / kEncodeWideThreads;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    encode_kernel<K, V, kEncodeWideThreads><<<(unsigned)blocks, kEncodeWideThreads, 0, stream>>>(a, tab);
+  } else {
+    const int64_t blocks = (items + kEncodeThreads - 1) / kEncodeThreads;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    encode_kernel<K, V, kEncodeThreads><<<(unsigned)blocks, kEncodeThreads, 0, stream>>>(a, tab);
+  }
   count_launch();
   return cudaGetLastError();
 }
