@@ -73,15 +73,19 @@ cudaError_t launch_one(const EncodeArgs& a, const EncodeTables& tab, cudaStream_
   // Rows that tile exactly into pieces of 768 columns (12 KB: a whole row of a 3x32x32 query) get CTAs of that
   // size: each CTA then reads and writes whole contiguous pieces of K and W rows, which HBM serves slightly
   // better (+0.8 % on workload 2) than the 4 KB pieces of 256-thread CTAs.
-  if (VecOps<V>::kLanes == 4 && Dv % kEncodeWideThreads == 0) {
-    const int64_t blocks = items / kEncodeWideThreads;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    encode_kernel<K, V, kEncodeWideThreads><<<(unsigned)blocks, kEncodeWideThreads, 0, stream>>>(a, tab);
-  } else {
-    const int64_t blocks = (items + kEncodeThreads - 1) / kEncodeThreads;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    encode_kernel<K, V, kEncodeThreads><<<(unsigned)blocks, kEncodeThreads, 0, stream>>>(a, tab);
+  // (K <= 16: beyond that 768 threads do not leave a thread enough registers for its K inputs)
+  if constexpr (VecOps<V>::kLanes == 4 && K <= 16) {
+    if (Dv % kEncodeWideThreads == 0) {
+      const int64_t blocks = items / kEncodeWideThreads;
+      if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+      encode_kernel<K, V, kEncodeWideThreads><<<(unsigned)blocks, kEncodeWideThreads, 0, stream>>>(a, tab);
+      count_launch();
+      return cudaGetLastError();
+    }
   }
+  const int64_t blocks = (items + kEncodeThreads - 1) / kEncodeThreads;
+  if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+  encode_kernel<K, V, kEncodeThreads><<<(unsigned)blocks, kEncodeThreads, 0, stream>>>(a, tab);
   count_launch();
   return cudaGetLastError();
 }

@@ -66,6 +66,9 @@ ENCODE_SHAPES = [
     (31, 2, 2, 4),
     (5, 32, 2, 516),
     (7, 9, 300, 4),      # D = 4: one column per group, many groups per block
+    (16, 20, 5, 3072),   # rows of 768 float4 columns: whole-row CTAs of 768 threads (K <= 16)
+    (3, 7, 2, 6144),     # two such CTAs per row, coincident nodes
+    (20, 24, 3, 3072),   # K > 16: stays on 256-thread CTAs
 ]
 
 
