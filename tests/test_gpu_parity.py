@@ -424,9 +424,12 @@ def test_staged_and_register_decoders_agree_bitwise_on_sums_order():
 
 
 @pytest.mark.parametrize("K,W,C,G", [(8, 12, 10, 1000), (8, 24, 10, 333), (4, 5, 10, 7), (3, 7, 9, 130), (1, 2, 1, 50),
-                                     (32, 32, 32, 21), (16, 24, 31, 64), (2, 5, 2, 257), (12, 20, 17, 90), (5, 9, 4, 3)])
+                                     (32, 32, 32, 21), (16, 24, 31, 64), (2, 5, 2, 257), (12, 20, 17, 90), (5, 9, 4, 3),
+                                     (8, 12, 100, 500), (16, 24, 128, 70), (16, 24, 256, 33), (12, 20, 36, 100), (5, 9, 64, 41),
+                                     (3, 7, 20, 50), (8, 12, 500, 9), (16, 24, 508, 5), (32, 32, 64, 6), (2, 5, 102, 77)])
 def test_short_payload_decoder_against_oracle_and_register_decoder(K, W, C, G):
-    """Dense buffers with at most 32 classes take the thread-per-query kernel.  It adds the same terms in the same
+    """Dense buffers with up to a few hundred classes take the thread-per-(query, chunk of classes) kernel
+    (a few shapes here fall outside it on purpose and must still be right).  It adds the same terms in the same
     order as the thread-per-class kernel: equal to the last bit, absent rows (NaN here) never used, both sign
     rules, coincident nodes ((K, W) = (3, 7), (1, 2) and (2, 5) have them), group counts that leave a ragged last CTA."""
     rng = np.random.default_rng(K * 100 + C)
