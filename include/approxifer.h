@@ -260,7 +260,7 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
                              float* w, int32_t* idx, int32_t* n, void* cuda_stream);
 
 /*
- * Test / tuning hook for the wide-payload decoder (C >= 512, 128-bit path,
+ * Test / tuning hook for the wide-payload decoder (C >= 128, 128-bit path,
  * default sign), which stages the rows of present workers through shared memory
  * with bulk asynchronous copies.  stages: 0 (as many as fit, at most 4) or an
  * upper bound >= 2 on the ring depth; ctas_per_sm: 0 (automatic) or an upper

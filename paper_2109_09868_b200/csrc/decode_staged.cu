@@ -402,6 +402,7 @@ cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t
 }
 
 constexpr int kWholeMaxK = 16;  // most queries one thread forms (SPLIT = 1)
+constexpr int kStagedMinC = 128;
 
 // Columns per work item.  Long contiguous pieces are what HBM likes: with 256 columns an item of workload 4
 // (rows of 250 float4) is whole rows -- one 4000-byte copy per present worker instead of two copies of about 2 KB
@@ -422,8 +423,9 @@ bool fits_256(const DecodeArgs& a) {
 
 template <int KT, int SPLIT>
 int auto_cols(const DecodeArgs& a) {
-  if (!fits_256<KT, SPLIT>(a)) return 128;
   const int64_t Cv = a.C / 4;
+  if (Cv <= 64) return 64;  // short rows: small items, up to four CTAs per SM
+  if (!fits_256<KT, SPLIT>(a)) return 128;
   const int64_t waste256 = (Cv + 255) / 256 * 256 - Cv, waste128 = (Cv + 127) / 128 * 128 - Cv;
   return waste256 <= waste128 ? 256 : 128;
 }
@@ -458,13 +460,15 @@ void decode_staged_config(int stages, int ctas_per_sm, int disable, int cols, in
   g_cfg_cols = cols;
 }
 
-// Wide rows on the 128-bit path.  Narrower payloads, and the (K, W) pairs in which some alpha_j equals some
-// beta_i (the row-copy case), stay on the register-staged kernel.
+// Rows of at least 128 floats on the 128-bit path (measured against the other two decoders on 3 GB problems,
+// K = 8 .. 16: 3.4-4.1 TB/s at C = 128, 4.9-5.9 TB/s from C = 200 on, where they reach 2.1-3.8 TB/s; below 128 they
+// are as fast or faster).  Narrower payloads, and the (K, W) pairs in which some alpha_j equals some beta_i (the
+// row-copy case), stay on the other kernels.
 bool decode_staged_eligible(const DecodeArgs& a) {
   if (g_cfg_disable) return false;
   const bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&
                    a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
-  if (!(vec && a.C >= 512)) return false;
+  if (!(vec && a.C >= kStagedMinC)) return false;
   for (int j = 0; j < a.K; ++j)
     for (int i = 0; i < a.W; ++i)
       if (nodes_coincide(a.K, a.W, j, i)) return false;

@@ -371,6 +371,10 @@ STAGED_SHAPES = [
     (32, 32, 9, 1028, 0),     # largest K and W
     (7, 13, 50, 516, 0),      # odd K: the two halves own 4 and 3 queries
     (1, 2, 20, 640, 0),       # K = 1: the second half of the CTA owns nothing
+    (16, 24, 90, 128, 0),     # shortest rows that take the staged path: 32 of 64 columns of an item in use
+    (8, 12, 70, 200, 0),      # 50 columns
+    (12, 20, 33, 256, 0),     # exactly one 64-column item per group
+    (16, 24, 40, 400, 0),     # 100 columns: 128-column items
 ]
 
 
