@@ -260,12 +260,12 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
                              float* w, int32_t* idx, int32_t* n, void* cuda_stream);
 
 /*
- * Test / tuning hook for the wide-payload decoder (C >= 96, 128-bit path,
+ * Test / tuning hook for the wide-payload decoder (C >= 64, 128-bit path,
  * default sign), which stages the rows of present workers through shared memory
  * with bulk asynchronous copies.  stages: 0 (as many as fit, at most 4) or an
  * upper bound >= 2 on the ring depth; ctas_per_sm: 0 (automatic) or an upper
  * bound; disable != 0 routes every decode through the register-staged kernel;
- * cols: 0 (automatic), 32 (split 2 only), 64, 128 or 256 16-byte columns per work item (256 needs split 1 or 2 and a
+ * cols: 0 (automatic), 16 or 32 (split 2 only), 64, 128 or 256 16-byte columns per work item (256 needs split 1 or 2 and a
  * ring that fits in shared memory, else 128 is used); split: 0 (automatic), 1 (K <= 16, 256 columns), 2 or 4
  * thread groups sharing the K queries of a column.
  * Process-wide, not thread-safe; results are bit-identical for every setting.

@@ -127,7 +127,7 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
 }
 
 int approxifer_debug_decode_config(int stages, int ctas_per_sm, int disable, int cols, int split) {
-  if (stages < 0 || stages == 1 || ctas_per_sm < 0 || (cols != 0 && cols != 32 && cols != 64 && cols != 128 && cols != 256) ||
+  if (stages < 0 || stages == 1 || ctas_per_sm < 0 || (cols != 0 && cols != 16 && cols != 32 && cols != 64 && cols != 128 && cols != 256) ||
       (split != 0 && split != 1 && split != 2 && split != 4))
     return APPROXIFER_E_PARAM;
   decode_staged_config(stages, ctas_per_sm, disable, cols, split);

@@ -227,10 +227,10 @@ bool decode_small_eligible(const DecodeArgs& a) {
   if (p.cp == 0 || a.K * p.nch > kSmallThreads) return false;
   // Where it pays (measured on 3 GB problems against the per-column kernel, K = 4 .. 24, C = 10 .. 400): short
   // rows, where the per-column kernel redoes the weights for every column (1.2-2.1x at C <= 36), and many
-  // queries, where that kernel's K accumulators per thread cost occupancy (1.2-1.7x at K >= 14, C < 96; from 96
+  // queries, where that kernel's K accumulators per thread cost occupancy (1.2-1.7x at K >= 14, C < 64; from 64
   // on the bulk-copy staged kernel takes over).
-  // Elsewhere below 96 the per-column kernel is as fast or faster (both reach only 2-3.6 TB/s there).
-  if (!(a.C <= 36 || (a.K >= 14 && a.C < 96))) return false;
+  // Elsewhere below 64 the per-column kernel is as fast or faster (both reach 3-3.5 TB/s there).
+  if (!(a.C <= 36 || (a.K >= 14 && a.C < 64))) return false;
   return groups_per_cta(a, p) >= 1;
 }
 

@@ -101,7 +101,7 @@ constexpr int kTableOff = 128;  // float rg[W][K] after the mbarriers and the ab
 __host__ __device__ constexpr int slots_off(int W, int K) { return (kTableOff + W * (K | 1) * 4 + 127) / 128 * 128; }
 __host__ __device__ constexpr int slot_bytes(int W, int KT, int SPLIT, int COLS) { return meta_bytes(W, KT, SPLIT) + W * COLS * 16; }
 __host__ __device__ constexpr int min_ctas(int KT, int threads) {
-  return KT > 8 ? 1 : (threads <= 96 ? 6 : (threads <= 160 ? 4 : (threads <= 288 ? 2 : 1)));
+  return KT > 8 ? 1 : (threads <= 64 ? 10 : (threads <= 96 ? 6 : (threads <= 160 ? 4 : (threads <= 288 ? 2 : 1))));
 }
 
 // Shared memory: full[4] empty[4] mbarriers, abort flag | rg[W][K] | S slots, each = item block + W rows of COLS*16 B.
@@ -404,7 +404,7 @@ cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t
 }
 
 constexpr int kWholeMaxK = 16;  // most queries one thread forms (SPLIT = 1)
-constexpr int kStagedMinC = 96;
+constexpr int kStagedMinC = 64;
 
 // Columns per work item.  Long contiguous pieces are what HBM likes: with 256 columns an item of workload 4
 // (rows of 250 float4) is whole rows -- one 4000-byte copy per present worker instead of two copies of about 2 KB
@@ -426,6 +426,7 @@ bool fits_256(const DecodeArgs& a) {
 template <int KT, int SPLIT>
 int auto_cols(const DecodeArgs& a) {
   const int64_t Cv = a.C / 4;
+  if (Cv <= 16 && SPLIT == 2) return 16;  // the shortest rows: one compute warp and one producer warp per CTA
   if (Cv <= 32 && SPLIT == 2) return 32;  // short rows: small items, six CTAs per SM
   if (Cv <= 64) return 64;
   if (!fits_256<KT, SPLIT>(a)) return 128;
@@ -442,9 +443,10 @@ cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cu
       int cols = g_cfg_cols ? g_cfg_cols : auto_cols<KT, SPLIT>(a);
       if (cols == 256 && !fits_256<KT, SPLIT>(a)) cols = 128;  // (a forced setting that cannot be honoured)
       if constexpr (SPLIT == 2) {
+        if (cols == 16) return launch_kt<KT, 16, SPLIT>(a, tab, stream);
         if (cols == 32) return launch_kt<KT, 32, SPLIT>(a, tab, stream);
       }
-      if (cols == 64 || cols == 32) return launch_kt<KT, 64, SPLIT>(a, tab, stream);
+      if (cols == 64 || cols == 32 || cols == 16) return launch_kt<KT, 64, SPLIT>(a, tab, stream);
       if constexpr (SPLIT == 2 && KT <= 8) {
         if (cols == 256) return launch_kt<KT, 256, SPLIT>(a, tab, stream);
       }
@@ -466,10 +468,10 @@ void decode_staged_config(int stages, int ctas_per_sm, int disable, int cols, in
   g_cfg_cols = cols;
 }
 
-// Rows of at least 96 floats on the 128-bit path (measured against the other two decoders on 3 GB problems,
-// K = 8 .. 16: 3.9-4.5 TB/s at C = 100, 5.0-5.6 TB/s at C = 128, 4.9-5.9 TB/s from C = 200 on, where they reach
-// 2.1-3.8 TB/s; at C = 64 they are faster).  Narrower payloads, and the (K, W) pairs in which some alpha_j equals
-// some beta_i (the row-copy case), stay on the other kernels.
+// Rows of at least 64 floats on the 128-bit path (measured against the other two decoders on 3 GB problems,
+// K = 8 .. 16: 3.6-4.9 TB/s at C = 64, 3.8-4.5 TB/s at C = 96-100, 5.0-5.7 TB/s at C = 128, 4.9-5.9 TB/s from
+// C = 200 on, where they reach 2.1-3.8 TB/s; at C = 40-48 they are as fast or faster).  Narrower payloads, and
+// the (K, W) pairs in which some alpha_j equals some beta_i (the row-copy case), stay on the other kernels.
 bool decode_staged_eligible(const DecodeArgs& a) {
   if (g_cfg_disable) return false;
   const bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&

@@ -374,6 +374,8 @@ STAGED_SHAPES = [
     (16, 24, 90, 128, 0),     # one 32-column item per group
     (12, 20, 75, 100, 0),     # 25 of 32 columns in use (the shortest rows that take the staged path have 96 floats)
     (6, 9, 51, 96, 0),
+    (8, 12, 64, 64, 0),       # the shortest rows that take the staged path: 16-column items, one compute warp
+    (5, 10, 40, 80, 0),
     (8, 12, 70, 200, 0),      # 50 columns
     (12, 20, 33, 256, 0),     # exactly one 64-column item per group
     (16, 24, 40, 400, 0),     # 100 columns: 128-column items
@@ -382,7 +384,7 @@ STAGED_SHAPES = [
 
 @pytest.mark.parametrize("stages,ctas,cols,split", [(0, 0, 0, 0), (2, 0, 128, 2), (3, 1, 128, 4), (4, 1, 64, 2), (2, 4, 64, 4), (0, 2, 64, 4),
                                                         (0, 0, 256, 2), (2, 1, 256, 0), (0, 0, 128, 0), (0, 0, 0, 1), (0, 0, 0, 2), (0, 0, 32, 2),
-                                                        (3, 0, 32, 0)])
+                                                        (3, 0, 32, 0), (0, 0, 16, 2)])
 def test_staged_decoder_matches_oracle_in_every_configuration(stages, ctas, cols, split):
     try:
         ap.debug_decode_config(stages, ctas, 0, cols, split)
