@@ -450,7 +450,6 @@ cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cu
       if constexpr (SPLIT == 2 && KT <= 8) {
         if (cols == 256) return launch_kt<KT, 256, SPLIT>(a, tab, stream);
       }
-      if constexpr (SPLIT == 1) return launch_kt<KT, 256, 1>(a, tab, stream);  // (the only single-group shape)
       return launch_kt<KT, 128, SPLIT>(a, tab, stream);
     }
     return dispatch_kt<SPLIT, KT + 1>(kt, a, tab, stream);
