@@ -25,9 +25,10 @@
  *     the legacy default stream) and the call returns without synchronising.
  *     The library never allocates device memory (its image contains one fixed
  *     staging array, see approxifer_encode_host_static), keeps no per-call
- *     state (only an immutable host-side cache of the node tables of each
- *     (K, W) seen) and may be called from several host threads on different
- *     streams.
+ *     state and no setting (only immutable host-side caches: the node tables
+ *     of each (K, W) seen, the current device's multiprocessor count and
+ *     shared-memory size) and may be called from several host threads on
+ *     different streams.
  *   - 16-byte aligned bases with D (or C) and all strides multiples of 4 take
  *     the 128-bit fast path; anything else runs a slower element-wise GPU
  *     path.  There is no CPU fallback.
@@ -72,6 +73,14 @@ extern "C" {
 #define APPROXIFER_ST_LOCATE_UNDERDETERMINED 4u /* locate: fewer than 2(K+E) workers present; nothing located */
 #define APPROXIFER_ST_NONFINITE 8u              /* locate: some Q(beta_i) was not finite (ranked as +inf) */
 
+/*
+ * One params struct serves a whole encode -> locate -> decode pipeline: every entry point reads the fields
+ * that concern it and ignores the rest.  E is ignored by encode and decode.  APPROXIFER_SIGN_WORKER_INDEX
+ * concerns the decoders only (approxifer_decode, approxifer_decode_host, step 2 of approxifer_locate_decode);
+ * APPROXIFER_LOCATE_HOMOGENEOUS concerns the locators only (approxifer_locate, approxifer_locate_host, step 1 of
+ * approxifer_locate_decode) -- approxifer_decode_rational always uses Q_0 = 1, as Algorithm 3 prints it, and the
+ * encoders have no flag.  A bit that no entry point defines is APPROXIFER_E_PARAM everywhere.
+ */
 typedef struct approxifer_params {
   int32_t K;      /* 1..32 queries per group */
   int32_t W;      /* 2..32 workers (paper: N+1) */
@@ -235,8 +244,11 @@ int approxifer_locate_host(const approxifer_params* params, int64_t G, int64_t C
  * and nothing is enqueued.
  *
  * The first call on each device looks up the array's device address (one
- * runtime query, no allocation); make that first call before starting any
- * stream capture on that device.  All calls on a device share the one array,
+ * runtime query, no allocation) and remembers it for the life of the process;
+ * make that first call before starting any stream capture on that device.
+ * `cuda_stream` must belong to the device that is current during the call, and
+ * the entry point must not be used again after that device has been reset
+ * (cudaDeviceReset): the remembered address is not looked up a second time.  All calls on a device share the one array,
  * which keeps the previous call's bytes (nothing in it needs clearing: each
  * call overwrites what it later reads).  Two calls whose GPU work can overlap
  * -- different streams without an ordering between them, or several host
@@ -260,25 +272,37 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
                              float* w, int32_t* idx, int32_t* n, void* cuda_stream);
 
 /*
- * Test / tuning hook for the wide-payload decoder (C >= 64, 128-bit path,
- * default sign), which stages the rows of present workers through shared memory
- * with bulk asynchronous copies.  stages: 0 (as many as fit, at most 4) or an
- * upper bound >= 2 on the ring depth; ctas_per_sm: 0 (automatic) or an upper
- * bound; disable != 0 routes every decode through the register-staged kernel;
- * cols: 0 (automatic), 16 or 32 (split 2 only), 64, 128 or 256 16-byte columns per work item (256 needs split 1 or 2 and a
- * ring that fits in shared memory, else 128 is used); split: 0 (automatic), 1 (K <= 16, 256 columns), 2 or 4
- * thread groups sharing the K queries of a column.
- * Process-wide, not thread-safe; results are bit-identical for every setting.
+ * Test / tuning hooks (not on the hot path): approxifer_decode and approxifer_locate with the choice of kernel
+ * and its launch plan given PER CALL.  The library itself keeps no such setting: these entry points change
+ * nothing for any other call or thread.  Results are bit-identical for every setting (Section 3, "ApproxIFER
+ * Decoding", steps 1 and 2, exactly as in the two entry points they shadow).
+ *
+ * `tuning` (HOST pointer, read during the call; NULL = all automatic), every field 0 = automatic:
+ *   kernel       1: route the call through the per-column register-staged kernel whatever the shape
+ *   stages       bulk-copy staged kernel (rows of >= 64 floats on the 128-bit path): upper bound >= 2 on the ring depth
+ *   ctas_per_sm  ... upper bound on resident CTAs per SM
+ *   cols         ... 16, 32 (split 2 only), 64, 128 or 256 16-byte columns per work item (256 needs split 1 or 2
+ *                and a ring that fits in shared memory, else 128 is used)
+ *   split        ... 1 (K <= 16, 256 columns), 2 or 4 thread groups sharing the K queries of a column
+ * APPROXIFER_E_PARAM for any other value.
+ *
+ * force_warp_kernel != 0 routes the locate through the warp-per-group kernel, which otherwise serves only
+ * K+E > 15 (smaller K+E use the thread-per-class kernel).  Both follow Algorithm 2 and return the same sets.
  */
-int approxifer_debug_decode_config(int stages, int ctas_per_sm, int disable, int cols, int split);
-
-/*
- * Test hook for the locator: force_warp_kernel != 0 routes every locate through the
- * warp-per-group kernel, which otherwise serves only K+E > 15 (smaller K+E use the
- * thread-per-class kernel).  Both follow Algorithm 2 and return the same sets.
- * Process-wide, not thread-safe.
- */
-int approxifer_debug_locate_config(int force_warp_kernel);
+typedef struct approxifer_decode_tuning {
+  int32_t kernel, stages, ctas_per_sm, cols, split;
+} approxifer_decode_tuning;
+int approxifer_debug_decode(const approxifer_params* params, int64_t G, int64_t C,
+                            const float* Yt, int64_t yt_gstride, int64_t yt_rstride,
+                            const uint32_t* mask,
+                            float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                            int32_t* n_used, uint32_t* status,
+                            const approxifer_decode_tuning* tuning, void* cuda_stream);
+int approxifer_debug_locate(const approxifer_params* params, int64_t G, int64_t C,
+                            const float* Yt, int64_t yt_gstride, int64_t yt_rstride,
+                            const uint32_t* mask,
+                            int32_t* adv, uint32_t* trusted_mask, uint32_t* status,
+                            int force_warp_kernel, void* cuda_stream);
 
 /*
  * Every wait on an asynchronous copy inside the kernels is bounded.  Returns how

@@ -18,8 +18,8 @@ from .binding import (  # noqa: F401
     approxifer_locate,
     approxifer_locate_decode,
     approxifer_params,
-    debug_decode_config,
-    debug_locate_config,
+    approxifer_decode_tuning,
+    decode_tuning,
     device_wait_timeouts,
     launch_count,
     library_path,

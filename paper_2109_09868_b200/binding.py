@@ -34,9 +34,9 @@ EXPORTS = (
     "approxifer_strerror",
     "approxifer_version",
     "approxifer_launch_count",
-    "approxifer_debug_decode_config",
+    "approxifer_debug_decode",
     "approxifer_device_wait_timeouts",
-    "approxifer_debug_locate_config",
+    "approxifer_debug_locate",
     "approxifer_encode_host",
     "approxifer_decode_host",
     "approxifer_locate_host",
@@ -46,6 +46,10 @@ EXPORTS = (
 
 class approxifer_params(ctypes.Structure):
     _fields_ = [("K", c_int32), ("W", c_int32), ("E", c_int32), ("flags", c_uint32)]
+
+
+class approxifer_decode_tuning(ctypes.Structure):
+    _fields_ = [("kernel", c_int32), ("stages", c_int32), ("ctas_per_sm", c_int32), ("cols", c_int32), ("split", c_int32)]
 
 
 class ApproxiferError(RuntimeError):
@@ -97,11 +101,13 @@ def load() -> ctypes.CDLL:
     lib.approxifer_strerror.restype = c_char_p
     lib.approxifer_version.restype = c_int
     lib.approxifer_launch_count.restype = c_int64
-    lib.approxifer_debug_decode_config.argtypes = [c_int, c_int, c_int, c_int, c_int]
-    lib.approxifer_debug_decode_config.restype = c_int
+    lib.approxifer_debug_decode.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_int64,
+                                            c_int64, c_void_p, c_void_p, POINTER(approxifer_decode_tuning), c_void_p]
+    lib.approxifer_debug_decode.restype = c_int
     lib.approxifer_device_wait_timeouts.restype = c_int64
-    lib.approxifer_debug_locate_config.argtypes = [c_int]
-    lib.approxifer_debug_locate_config.restype = c_int
+    lib.approxifer_debug_locate.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
+                                            c_void_p, c_int, c_void_p]
+    lib.approxifer_debug_locate.restype = c_int
     c_size_t = ctypes.c_size_t
     lib.approxifer_encode_host.argtypes = [pp, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_size_t, POINTER(c_void_p), c_int]
     lib.approxifer_encode_host.restype = c_int
@@ -130,14 +136,9 @@ def launch_count() -> int:
     return int(load().approxifer_launch_count())
 
 
-def debug_decode_config(stages: int = 0, ctas_per_sm: int = 0, disable: int = 0, cols: int = 0, split: int = 0) -> None:
-    rc = load().approxifer_debug_decode_config(int(stages), int(ctas_per_sm), int(disable), int(cols), int(split))
-    if rc != OK:
-        raise ApproxiferError(rc, "approxifer_debug_decode_config")
-
-
-def debug_locate_config(force_warp_kernel: int = 0) -> None:
-    load().approxifer_debug_locate_config(int(force_warp_kernel))
+def decode_tuning(kernel: int = 0, stages: int = 0, ctas_per_sm: int = 0, cols: int = 0, split: int = 0) -> approxifer_decode_tuning:
+    """Per-call kernel choice / launch plan for approxifer_decode(..., tuning=...) (tests and tuning only)."""
+    return approxifer_decode_tuning(int(kernel), int(stages), int(ctas_per_sm), int(cols), int(split))
 
 
 def device_wait_timeouts() -> int:
@@ -188,8 +189,10 @@ def approxifer_encode(params: approxifer_params, X: torch.Tensor, Xt: Optional[t
 
 
 def approxifer_decode(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, Yhat: Optional[torch.Tensor] = None,
-                      n_used: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """Yt [G][W][C], mask [G] (int32 tensor holding the uint32 bit patterns) -> Yhat [G][K][C]."""
+                      n_used: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, stream=None,
+                      tuning: Optional[approxifer_decode_tuning] = None) -> torch.Tensor:
+    """Yt [G][W][C], mask [G] (int32 tensor holding the uint32 bit patterns) -> Yhat [G][K][C].
+    With `tuning` the call goes through approxifer_debug_decode (same result, chosen kernel / launch plan)."""
     G, W, C = Yt.shape
     if Yhat is None:
         Yhat = torch.empty((G, params.K, C), device=Yt.device, dtype=torch.float32)
@@ -198,17 +201,24 @@ def approxifer_decode(params: approxifer_params, Yt: torch.Tensor, mask: torch.T
     if Yhat.shape[0] != G or Yhat.shape[2] != C:
         raise ValueError("Yhat must be [G][K][C]")
     mp = _vec(mask, torch.int32, G, "mask")
-    rc = load().approxifer_decode(ctypes.byref(params), G, C, yp, yg, yr, mp, op, og, orr,
-                                  _vec(n_used, torch.int32, G, "n_used"), _vec(status, torch.int32, G, "status"),
-                                  _stream_ptr(stream))
+    if tuning is not None:
+        rc = load().approxifer_debug_decode(ctypes.byref(params), G, C, yp, yg, yr, mp, op, og, orr,
+                                            _vec(n_used, torch.int32, G, "n_used"), _vec(status, torch.int32, G, "status"),
+                                            ctypes.byref(tuning), _stream_ptr(stream))
+    else:
+        rc = load().approxifer_decode(ctypes.byref(params), G, C, yp, yg, yr, mp, op, og, orr,
+                                      _vec(n_used, torch.int32, G, "n_used"), _vec(status, torch.int32, G, "status"),
+                                      _stream_ptr(stream))
     if rc != OK:
         raise ApproxiferError(rc, "approxifer_decode")
     return Yhat
 
 
 def approxifer_locate(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, adv: Optional[torch.Tensor] = None,
-                      trusted_mask: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, stream=None):
-    """Yt [G][W][C], mask [G] -> (adv [G][E] int32, trusted_mask [G] int32 bit patterns)."""
+                      trusted_mask: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, stream=None,
+                      force_warp_kernel: bool = False):
+    """Yt [G][W][C], mask [G] -> (adv [G][E] int32, trusted_mask [G] int32 bit patterns).
+    force_warp_kernel (tests): through approxifer_debug_locate, on the warp-per-group kernel."""
     G, W, C = Yt.shape
     E = max(int(params.E), 0)
     if adv is None:
@@ -216,9 +226,13 @@ def approxifer_locate(params: approxifer_params, Yt: torch.Tensor, mask: torch.T
     if trusted_mask is None:
         trusted_mask = torch.empty((G,), device=Yt.device, dtype=torch.int32)
     yp, yg, yr = _payload(Yt, params.W, "Yt")
-    rc = load().approxifer_locate(ctypes.byref(params), G, C, yp, yg, yr, _vec(mask, torch.int32, G, "mask"),
-                                  _vec(adv, torch.int32, G * E, "adv"), _vec(trusted_mask, torch.int32, G, "trusted_mask"),
-                                  _vec(status, torch.int32, G, "status"), _stream_ptr(stream))
+    args = (ctypes.byref(params), G, C, yp, yg, yr, _vec(mask, torch.int32, G, "mask"),
+            _vec(adv, torch.int32, G * E, "adv"), _vec(trusted_mask, torch.int32, G, "trusted_mask"),
+            _vec(status, torch.int32, G, "status"))
+    if force_warp_kernel:
+        rc = load().approxifer_debug_locate(*args, 1, _stream_ptr(stream))
+    else:
+        rc = load().approxifer_locate(*args, _stream_ptr(stream))
     if rc != OK:
         raise ApproxiferError(rc, "approxifer_locate")
     return adv, trusted_mask

@@ -32,6 +32,20 @@ def nvcc() -> str:
     return exe
 
 
+MIN_CUDA = (12, 8)  # sm_100a needs CUDA 12.8; kernel parameter blocks above 4 KB (the weight tables) need 12.1
+
+
+def check_toolkit() -> None:
+    """Fails with a clear message when nvcc is older than the kernels need."""
+    import re
+
+    out = subprocess.run([nvcc(), "--version"], capture_output=True, text=True).stdout
+    m = re.search(r"release (\d+)\.(\d+)", out)
+    if m and (int(m.group(1)), int(m.group(2))) < MIN_CUDA:
+        raise RuntimeError("nvcc %s.%s is too old: the library needs CUDA %d.%d or later (sm_100a target, kernel "
+                           "parameter blocks of up to 32 KB)" % (m.group(1), m.group(2), *MIN_CUDA))
+
+
 def _deps_mtime() -> float:
     paths = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, "approxifer.h"), __file__]
     return max(os.path.getmtime(p) for p in paths)
@@ -59,6 +73,7 @@ def _compile(src: str, verbose: bool) -> str:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not is_stale():
         return LIB
+    check_toolkit()
     os.makedirs(OBJDIR, exist_ok=True)
     with concurrent.futures.ThreadPoolExecutor(max_workers=len(SOURCES)) as ex:
         objs = list(ex.map(lambda s: _compile(s, verbose), SOURCES))

@@ -13,6 +13,26 @@ std::atomic<long long> g_launches{0};
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+cudaError_t current_device_info(const DeviceInfo** out) {
+  static DeviceInfo info[kMaxDevices];
+  static std::atomic<int> ready[kMaxDevices];
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!ready[dev].load(std::memory_order_acquire)) {
+    // (two threads may both fill the entry: they write the same values)
+    DeviceInfo d;
+    d.ordinal = dev;
+    if ((e = cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&d.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev)) != cudaSuccess) return e;
+    info[dev] = d;
+    ready[dev].store(1, std::memory_order_release);
+  }
+  *out = &info[dev];
+  return cudaSuccess;
+}
+
 namespace {
 
 int check_kw(const approxifer_params* p) {
@@ -36,7 +56,42 @@ int from_cuda(cudaError_t e) { return e == cudaSuccess ? APPROXIFER_OK : APPROXI
 
 using namespace approxifer;
 
+namespace {
+int decode_checked(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
+                   int64_t yt_rstride, const uint32_t* mask, float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                   int32_t* n_used, uint32_t* status, const DecodeTuning& tune, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if ((rc = check_layout(G, C, yt_rstride))) return rc;
+  if ((rc = check_layout(G, C, yh_rstride))) return rc;
+  if (yt_gstride < 0 || yh_gstride < 0) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (Yt == nullptr || Yhat == nullptr || mask == nullptr) return APPROXIFER_E_NULL;
+  DecodeArgs a{Yt,         mask,       Yhat,       n_used, status, yt_gstride, yt_rstride,
+               yh_gstride, yh_rstride, G,          C,      params->K, params->W, params->flags, tune};
+  return from_cuda(launch_decode(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int locate_checked(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
+                   int64_t yt_rstride, const uint32_t* mask, int32_t* adv, uint32_t* trusted_mask, uint32_t* status,
+                   int force_warp_kernel, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if (params->E < 0) return APPROXIFER_E_RANGE;
+  if (params->E < 1 || 2 * (params->K + params->E) > params->W) return APPROXIFER_E_PARAM;
+  if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateAltMaxM) return APPROXIFER_E_PARAM;
+  if ((rc = check_layout(G, C, yt_rstride))) return rc;
+  if (yt_gstride < 0) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (Yt == nullptr || mask == nullptr || adv == nullptr || trusted_mask == nullptr) return APPROXIFER_E_NULL;
+  LocateArgs a{Yt, mask, adv, trusted_mask, status, yt_gstride, yt_rstride, G, C, params->K, params->W, params->E, params->flags};
+  a.force_warp_kernel = force_warp_kernel;
+  return from_cuda(launch_locate(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+}  // namespace
+
 extern "C" {
+
 
 int approxifer_encode(const approxifer_params* params, int64_t G, int64_t D, const float* X, int64_t x_gstride,
                       int64_t x_rstride, float* Xt, int64_t xt_gstride, int64_t xt_rstride, void* cuda_stream) {
@@ -54,32 +109,37 @@ int approxifer_encode(const approxifer_params* params, int64_t G, int64_t D, con
 int approxifer_decode(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
                       int64_t yt_rstride, const uint32_t* mask, float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
                       int32_t* n_used, uint32_t* status, void* cuda_stream) {
-  int rc = check_kw(params);
-  if (rc) return rc;
-  if ((rc = check_layout(G, C, yt_rstride))) return rc;
-  if ((rc = check_layout(G, C, yh_rstride))) return rc;
-  if (yt_gstride < 0 || yh_gstride < 0) return APPROXIFER_E_RANGE;
-  if (G == 0) return APPROXIFER_OK;
-  if (Yt == nullptr || Yhat == nullptr || mask == nullptr) return APPROXIFER_E_NULL;
-  DecodeArgs a{Yt,         mask,       Yhat,       n_used, status, yt_gstride, yt_rstride,
-               yh_gstride, yh_rstride, G,          C,      params->K, params->W, params->flags};
-  return from_cuda(launch_decode(a, static_cast<cudaStream_t>(cuda_stream)));
+  return decode_checked(params, G, C, Yt, yt_gstride, yt_rstride, mask, Yhat, yh_gstride, yh_rstride, n_used, status,
+                        DecodeTuning{}, cuda_stream);
+}
+
+int approxifer_debug_decode(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
+                            int64_t yt_rstride, const uint32_t* mask, float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                            int32_t* n_used, uint32_t* status, const approxifer_decode_tuning* tuning, void* cuda_stream) {
+  DecodeTuning t{};
+  if (tuning != nullptr) {
+    const int cols = tuning->cols, split = tuning->split;
+    if (tuning->kernel < 0 || tuning->kernel > 1 || tuning->stages < 0 || tuning->stages == 1 || tuning->ctas_per_sm < 0 ||
+        (cols != 0 && cols != 16 && cols != 32 && cols != 64 && cols != 128 && cols != 256) ||
+        (split != 0 && split != 1 && split != 2 && split != 4))
+      return APPROXIFER_E_PARAM;
+    t.kernel = tuning->kernel, t.stages = tuning->stages, t.ctas_per_sm = tuning->ctas_per_sm, t.cols = cols, t.split = split;
+  }
+  return decode_checked(params, G, C, Yt, yt_gstride, yt_rstride, mask, Yhat, yh_gstride, yh_rstride, n_used, status, t,
+                        cuda_stream);
 }
 
 int approxifer_locate(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
                       int64_t yt_rstride, const uint32_t* mask, int32_t* adv, uint32_t* trusted_mask, uint32_t* status,
                       void* cuda_stream) {
-  int rc = check_kw(params);
-  if (rc) return rc;
-  if (params->E < 0) return APPROXIFER_E_RANGE;
-  if (params->E < 1 || 2 * (params->K + params->E) > params->W) return APPROXIFER_E_PARAM;
-  if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateAltMaxM) return APPROXIFER_E_PARAM;
-  if ((rc = check_layout(G, C, yt_rstride))) return rc;
-  if (yt_gstride < 0) return APPROXIFER_E_RANGE;
-  if (G == 0) return APPROXIFER_OK;
-  if (Yt == nullptr || mask == nullptr || adv == nullptr || trusted_mask == nullptr) return APPROXIFER_E_NULL;
-  LocateArgs a{Yt, mask, adv, trusted_mask, status, yt_gstride, yt_rstride, G, C, params->K, params->W, params->E, params->flags};
-  return from_cuda(launch_locate(a, static_cast<cudaStream_t>(cuda_stream)));
+  return locate_checked(params, G, C, Yt, yt_gstride, yt_rstride, mask, adv, trusted_mask, status, 0, cuda_stream);
+}
+
+int approxifer_debug_locate(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
+                            int64_t yt_rstride, const uint32_t* mask, int32_t* adv, uint32_t* trusted_mask, uint32_t* status,
+                            int force_warp_kernel, void* cuda_stream) {
+  return locate_checked(params, G, C, Yt, yt_gstride, yt_rstride, mask, adv, trusted_mask, status, force_warp_kernel != 0,
+                        cuda_stream);
 }
 
 int approxifer_decode_rational(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
@@ -124,19 +184,6 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
   if (w == nullptr || (which == 1 && (idx == nullptr || n == nullptr))) return APPROXIFER_E_NULL;
   return from_cuda(launch_debug_weights(params->K, params->W, params->flags, mask, which, w, idx, n,
                                         static_cast<cudaStream_t>(cuda_stream)));
-}
-
-int approxifer_debug_decode_config(int stages, int ctas_per_sm, int disable, int cols, int split) {
-  if (stages < 0 || stages == 1 || ctas_per_sm < 0 || (cols != 0 && cols != 16 && cols != 32 && cols != 64 && cols != 128 && cols != 256) ||
-      (split != 0 && split != 1 && split != 2 && split != 4))
-    return APPROXIFER_E_PARAM;
-  decode_staged_config(stages, ctas_per_sm, disable, cols, split);
-  return APPROXIFER_OK;
-}
-
-int approxifer_debug_locate_config(int force_warp_kernel) {
-  locate_config(force_warp_kernel);
-  return APPROXIFER_OK;
 }
 
 int64_t approxifer_device_wait_timeouts(void) {

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdint>
 
 #include "tables.h"
@@ -25,6 +26,15 @@ struct EncodeArgs {
   int32_t K, W;
 };
 
+// Test / tuning choices of one decode call (all zero = automatic); see approxifer_debug_decode.
+struct DecodeTuning {
+  int32_t kernel = 0;       // 0 automatic, 1 the per-column register-staged kernel
+  int32_t stages = 0;       // bulk-copy staged kernel: upper bound on the ring depth
+  int32_t ctas_per_sm = 0;  // ... upper bound on resident CTAs per SM
+  int32_t cols = 0;         // ... 16-byte columns per work item
+  int32_t split = 0;        // ... thread groups sharing the K queries of a column
+};
+
 struct DecodeArgs {
   const float* Yt;
   const uint32_t* mask;
@@ -35,6 +45,7 @@ struct DecodeArgs {
   int64_t G, C;
   int32_t K, W;
   uint32_t flags;
+  DecodeTuning tune = {};
 };
 
 struct LocateArgs {
@@ -50,6 +61,7 @@ struct LocateArgs {
   // Algorithm 3 (rational decoding) only: where r(alpha_j) goes; NULL for the locator proper
   float* Yh = nullptr;
   int64_t o_gs = 0, o_rs = 0;
+  int32_t force_warp_kernel = 0;  // test hook: the warp-per-group kernel also where the thread-per-class one would run
 };
 
 // Each returns a cudaError_t from the launch (cudaSuccess if nothing to do).
@@ -62,22 +74,40 @@ cudaError_t launch_debug_weights(int K, int W, uint32_t flags, uint32_t mask, in
 // Wide-payload decoder (bulk-copy staged); see decode_staged.cu.
 bool decode_staged_eligible(const DecodeArgs& a);
 cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream);
-void decode_staged_config(int stages, int ctas_per_sm, int disable, int cols, int split);
 cudaError_t read_decode_wait_timeouts(unsigned int* out);
 
 // Short-payload decoder (C <= 32, dense buffers); see decode_small.cu.
 bool decode_small_eligible(const DecodeArgs& a);
 cudaError_t launch_decode_small(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream);
-void decode_small_config(int disable);
 
 // Thread-per-class locator for K+E <= kLocateRowsMaxM (locate_rows_impl.cuh); the warp-per-group kernel covers the rest.
 constexpr int kLocateRowsMaxM = 15;
 // ... and its alternative last steps (Algorithm 1's homogeneous system, Algorithm 3) for K+E <= kLocateAltMaxM
 constexpr int kLocateAltMaxM = 13;
 cudaError_t launch_locate_rows(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream);
-void locate_config(int force_warp_kernel);
 
 void count_launch(int n = 1);
+
+// What the launch planners need to know about the current device, asked once per device and process.
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+  int ordinal = -1;
+  int sms = 0;          // multiprocessors
+  int smem_per_sm = 0;  // shared memory per multiprocessor, bytes
+};
+cudaError_t current_device_info(const DeviceInfo** out);
+
+// Raises a kernel's dynamic shared-memory limit to `bytes` on device `dev` unless an earlier call already
+// did (one cache per kernel: instantiate with the kernel's own tag type).
+template <typename KernelTag, typename Kernel>
+cudaError_t ensure_dynamic_smem(Kernel kernel, int dev, int bytes) {
+  static std::atomic<int> granted[kMaxDevices];
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (bytes <= 48 * 1024 || bytes <= granted[dev].load(std::memory_order_acquire)) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) granted[dev].store(bytes, std::memory_order_release);
+  return e;
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -144,8 +144,6 @@ __global__ void __launch_bounds__(kSmallThreads) decode_small_kernel(const __gri
   }
 }
 
-bool g_small_disabled = false;
-
 // How a row of C classes is cut into per-thread chunks: CP classes each, V floats per shared-memory access.
 struct ChunkPlan {
   int cp = 0, v = 0, nch = 0;
@@ -189,8 +187,11 @@ cudaError_t launch_small(const DecodeArgs& a, const DecodeTables& tab, const Chu
   const int64_t blocks = (a.G + gpb - 1) / gpb;
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(decode_small_kernel<CP, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const DeviceInfo* di = nullptr;
+    cudaError_t e = current_device_info(&di);
     if (e != cudaSuccess) return e;
+    struct Tag {};
+    if ((e = ensure_dynamic_smem<Tag>(decode_small_kernel<CP, V>, di->ordinal, (int)smem)) != cudaSuccess) return e;
   }
   decode_small_kernel<CP, V><<<(unsigned)blocks, kSmallThreads, smem, stream>>>(a, tab, gpb, p.nch);
   count_launch();
@@ -215,12 +216,10 @@ cudaError_t dispatch_cp(const DecodeArgs& a, const DecodeTables& tab, const Chun
 
 }  // namespace
 
-void decode_small_config(int disable) { g_small_disabled = disable != 0; }
-
 // Dense buffers (rows and groups back to back), 16-byte aligned, a class count that cuts into chunks (see
 // plan_chunks), and room for at least one group per CTA.
 bool decode_small_eligible(const DecodeArgs& a) {
-  if (g_small_disabled) return false;
+  if (a.tune.kernel == 1) return false;
   if (a.y_rs != a.C || a.y_gs != (int64_t)a.W * a.C || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
   if (!aligned16(a.Yt) || !aligned16(a.Yh)) return false;
   const ChunkPlan p = plan_chunks(a.C);

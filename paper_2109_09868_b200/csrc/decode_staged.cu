@@ -21,7 +21,7 @@
 // starts the copies of the present rows; slots are handed over and back
 // through "full" / "empty" mbarriers, so producer and compute warps never meet
 // at a CTA-wide barrier.  Every wait is bounded.  Items are dealt round-robin
-// to the CTAs.  No cluster multicast is used.
+// to the CTAs.  Every copy targets the issuing CTA's own shared memory.
 #include "common.cuh"
 
 namespace approxifer {
@@ -362,12 +362,6 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
   }
 }
 
-int g_cfg_stages = 0;  // 0 = automatic; test / tuning hooks
-int g_cfg_ctas_per_sm = 0;
-int g_cfg_disable = 0;
-int g_cfg_cols = 0;
-int g_cfg_split = 0;
-
 template <int KT, int COLS, int SPLIT>
 cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream) {
   const int64_t Cv = a.C / 4;
@@ -376,28 +370,27 @@ cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t
   plan.n_items = a.G * plan.tiles;
   const int64_t slot = slot_bytes(a.W, KT, SPLIT, COLS);
 
-  int dev = 0, sms = 0, smem_sm = 0;
-  cudaError_t e = cudaGetDevice(&dev);
+  const DeviceInfo* di = nullptr;
+  cudaError_t e = current_device_info(&di);
   if (e != cudaSuccess) return e;
-  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-  if ((e = cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev)) != cudaSuccess) return e;
+  const int sms = di->sms, smem_sm = di->smem_per_sm;
   const int fixed = slots_off(a.W, a.K);
   // as many CTAs per SM as fit with a two-slot ring (at most 4 small or 2 large ones), then the ring as deep
   // as the rest allows
   int ctas = min_ctas(KT, SPLIT * COLS + 32);
-  if (g_cfg_ctas_per_sm > 0 && g_cfg_ctas_per_sm < ctas) ctas = g_cfg_ctas_per_sm;
+  if (a.tune.ctas_per_sm > 0 && a.tune.ctas_per_sm < ctas) ctas = a.tune.ctas_per_sm;
   while (ctas > 1 && (int64_t)ctas * (fixed + 2 * slot + 1024) > smem_sm) --ctas;
   int stages = (int)(((int64_t)smem_sm / ctas - 1024 - fixed) / slot);  // 1 KB per CTA is reserved
   if (stages < 2) return cudaErrorInvalidConfiguration;
   if (stages > kMaxStages) stages = kMaxStages;
-  if (g_cfg_stages >= 2 && g_cfg_stages < stages) stages = g_cfg_stages;
+  if (a.tune.stages >= 2 && a.tune.stages < stages) stages = a.tune.stages;
   plan.stages = stages;
   const size_t smem = (size_t)fixed + (size_t)stages * slot;
   int64_t grid = (int64_t)sms * ctas;
   if (grid > plan.n_items) grid = plan.n_items;
 
-  e = cudaFuncSetAttribute(decode_staged_kernel<KT, COLS, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
+  struct Tag {};
+  if ((e = ensure_dynamic_smem<Tag>(decode_staged_kernel<KT, COLS, SPLIT>, di->ordinal, (int)smem)) != cudaSuccess) return e;
   decode_staged_kernel<KT, COLS, SPLIT><<<(unsigned)grid, SPLIT * COLS + 32, smem, stream>>>(a, tab, plan);
   count_launch();
   return cudaGetLastError();
@@ -416,10 +409,9 @@ bool fits_256(const DecodeArgs& a) {
   // 544 threads (two thread groups) leave 112 registers each: enough for 8 queries per thread; a single thread
   // group of 256 carries up to 16
   if (SPLIT == 4 || (SPLIT == 2 && KT > 8) || (SPLIT == 1 && KT > kWholeMaxK)) return false;
-  int dev = 0, smem_sm = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
-    return false;
+  const DeviceInfo* di = nullptr;
+  if (current_device_info(&di) != cudaSuccess) return false;
+  const int smem_sm = di->smem_per_sm;
   return (int64_t)slots_off(a.W, a.K) + 2 * (int64_t)slot_bytes(a.W, KT, SPLIT, 256) + 1024 <= smem_sm;
 }
 
@@ -440,7 +432,7 @@ cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cu
     return cudaErrorInvalidValue;
   } else {
     if (kt == KT) {
-      int cols = g_cfg_cols ? g_cfg_cols : auto_cols<KT, SPLIT>(a);
+      int cols = a.tune.cols ? a.tune.cols : auto_cols<KT, SPLIT>(a);
       if (cols == 256 && !fits_256<KT, SPLIT>(a)) cols = 128;  // (a forced setting that cannot be honoured)
       if constexpr (SPLIT == 2) {
         if (cols == 16) return launch_kt<KT, 16, SPLIT>(a, tab, stream);
@@ -458,21 +450,12 @@ cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cu
 
 }  // namespace
 
-void decode_staged_config(int stages, int ctas_per_sm, int disable, int cols, int split) {
-  g_cfg_split = split;
-  g_cfg_stages = stages;
-  g_cfg_ctas_per_sm = ctas_per_sm;
-  g_cfg_disable = disable;
-  decode_small_config(disable);
-  g_cfg_cols = cols;
-}
-
 // Rows of at least 64 floats on the 128-bit path (measured against the other two decoders on 3 GB problems,
 // K = 8 .. 16: 3.6-4.9 TB/s at C = 64, 3.8-4.5 TB/s at C = 96-100, 5.0-5.7 TB/s at C = 128, 4.9-5.9 TB/s from
 // C = 200 on, where they reach 2.1-3.8 TB/s; at C = 40-48 they are as fast or faster).  Narrower payloads, and
 // the (K, W) pairs in which some alpha_j equals some beta_i (the row-copy case), stay on the other kernels.
 bool decode_staged_eligible(const DecodeArgs& a) {
-  if (g_cfg_disable) return false;
+  if (a.tune.kernel == 1) return false;
   const bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&
                    a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
   if (!(vec && a.C >= kStagedMinC)) return false;
@@ -495,7 +478,7 @@ cudaError_t dispatch_whole(const DecodeArgs& a, const DecodeTables& tab, cudaStr
     if (a.K == KT) {
       const int64_t Cv = a.C / 4;
       const int64_t waste256 = (Cv + 255) / 256 * 256 - Cv, waste128 = (Cv + 127) / 128 * 128 - Cv;
-      const bool want = g_cfg_split == 1 || (g_cfg_split == 0 && (g_cfg_cols == 0 || g_cfg_cols == 256) && waste256 <= waste128);
+      const bool want = a.tune.split == 1 || (a.tune.split == 0 && (a.tune.cols == 0 || a.tune.cols == 256) && waste256 <= waste128);
       *taken = want && fits_256<KT, 1>(a);
       return *taken ? launch_kt<KT, 256, 1>(a, tab, stream) : cudaSuccess;
     }
@@ -507,7 +490,7 @@ cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, c
   bool taken = false;
   const cudaError_t e = dispatch_whole<>(a, tab, stream, &taken);
   if (taken) return e;
-  if (g_cfg_split == 4) return dispatch_kt<4>((a.K + 3) / 4, a, tab, stream);
+  if (a.tune.split == 4) return dispatch_kt<4>((a.K + 3) / 4, a, tab, stream);
   return dispatch_kt<2>((a.K + 1) / 2, a, tab, stream);
 }
 

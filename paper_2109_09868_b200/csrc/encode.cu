@@ -11,6 +11,10 @@ namespace approxifer {
 
 namespace {
 
+// The weight table travels as a kernel parameter (constant bank): together with the arguments it must stay
+// within the 32,764 bytes a launch may pass (parameter blocks above 4 KB need CUDA 12.1 or later).
+static_assert(sizeof(EncodeArgs) + sizeof(EncodeTables) <= 32764, "encode kernel parameters exceed the launch limit");
+
 constexpr int kEncodeThreads = 256;
 constexpr int kEncodeWideThreads = 768;
 

@@ -240,9 +240,12 @@ __global__ void __launch_bounds__(kLocateThreads) locate_kernel(const __grid_con
 template <int NMAX, int M>
 cudaError_t launch_nm(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream) {
   const size_t smem = sizeof(WarpSmem<NMAX, M>) * kLocateWarps;
-  if (smem > 48 * 1024) {  // opt in to more than the default dynamic shared memory (per device, idempotent)
-    cudaError_t e = cudaFuncSetAttribute(locate_kernel<NMAX, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (smem > 48 * 1024) {  // opt in to more than the default dynamic shared memory (once per device)
+    const DeviceInfo* di = nullptr;
+    cudaError_t e = current_device_info(&di);
     if (e != cudaSuccess) return e;
+    struct Tag {};
+    if ((e = ensure_dynamic_smem<Tag>(locate_kernel<NMAX, M>, di->ordinal, (int)smem)) != cudaSuccess) return e;
   }
   const int64_t blocks = (a.G + kLocateWarps - 1) / kLocateWarps;
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
@@ -262,11 +265,7 @@ cudaError_t dispatch_m(int m, const LocateArgs& a, const LocateTables& tab, cuda
   }
 }
 
-int g_force_warp_kernel = 0;  // test hook
-
 }  // namespace
-
-void locate_config(int force_warp_kernel) { g_force_warp_kernel = force_warp_kernel; }
 
 cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
@@ -274,7 +273,7 @@ cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream) {
   const int m = a.K + a.E;
   // (the homogeneous form and Algorithm 3 exist in the thread-per-class kernel only; the entry points have checked K+E)
   const bool alt = (a.flags & kFlagLocateHomogeneous) || a.Yh != nullptr;
-  if (alt ? m <= kLocateAltMaxM : (m <= kLocateRowsMaxM && !g_force_warp_kernel))
+  if (alt ? m <= kLocateAltMaxM : (m <= kLocateRowsMaxM && !a.force_warp_kernel))
     return launch_locate_rows(a, tab, stream);
   if (a.W <= 8) return dispatch_m<8>(m, a, tab, stream);
   if (a.W <= 16) return dispatch_m<16>(m, a, tab, stream);

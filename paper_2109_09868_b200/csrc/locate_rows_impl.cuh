@@ -17,6 +17,8 @@
 // (ties to the lower worker) and votes with shared-memory atomics; a warp per group elects the E most voted
 // workers.  Everything runs in fp64.
 #pragma once
+#include <type_traits>
+
 #include "common.cuh"
 #include "locate_common.cuh"
 
@@ -25,6 +27,9 @@ namespace approxifer {
 namespace {
 
 using namespace locate_detail;
+
+static_assert(sizeof(LocateArgs) + sizeof(LocateTables) + sizeof(LocateBasis) + 16 <= 32764,
+              "locator kernel parameters exceed the launch limit (blocks above 4 KB need CUDA 12.1 or later)");
 
 constexpr int kRowsThreads = 128;
 constexpr int kRowsWarps = kRowsThreads / 32;
@@ -573,20 +578,24 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
   const size_t smem = (size_t)gpb * per_group + y_bytes;
   const int64_t blocks = (a.G + gpb - 1) / gpb;
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-  auto run = [&](auto kernel) -> cudaError_t {
+  auto run = [&](auto mode) -> cudaError_t {
+    constexpr int MODE = decltype(mode)::value;
     if (smem > 48 * 1024) {
-      cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      const DeviceInfo* di = nullptr;
+      cudaError_t e = current_device_info(&di);
       if (e != cudaSuccess) return e;
+      struct Tag {};
+      if ((e = ensure_dynamic_smem<Tag>(locate_rows_kernel<NMAX, M, MODE>, di->ordinal, (int)smem)) != cudaSuccess) return e;
     }
-    kernel<<<(unsigned)blocks, kRowsThreads, smem, stream>>>(a, tab, locate_basis(a.W, M), (int)gpb);
+    locate_rows_kernel<NMAX, M, MODE><<<(unsigned)blocks, kRowsThreads, smem, stream>>>(a, tab, locate_basis(a.W, M), (int)gpb);
     count_launch();
     return cudaGetLastError();
   };
   if constexpr (M <= kLocateAltMaxM) {
-    if (a.Yh != nullptr) return run(locate_rows_kernel<NMAX, M, kModeRational>);
-    if (a.flags & kFlagLocateHomogeneous) return run(locate_rows_kernel<NMAX, M, kModeHomogeneous>);
+    if (a.Yh != nullptr) return run(std::integral_constant<int, kModeRational>{});
+    if (a.flags & kFlagLocateHomogeneous) return run(std::integral_constant<int, kModeHomogeneous>{});
   }
-  return run(locate_rows_kernel<NMAX, M, kModeLocate>);
+  return run(std::integral_constant<int, kModeLocate>{});
 }
 
 template <int NMAX, int M = 2>

@@ -9,8 +9,9 @@
 // exits, whether or not this entry point is ever called.
 //
 // The staging area keeps whatever the previous call left in it.  Nothing in it has to start at zero: the
-// host-to-device copy overwrites the query part completely before the kernel reads it, and the kernel
-// writes every element of the coded-query part that the device-to-host copy then reads.
+// host-to-device copy writes every query element the kernel reads, and the kernel writes every element of the
+// coded-query part that the device-to-host copy then reads.  (When D is not a multiple of 4 the rows are
+// padded to whole 16-byte columns; the pad elements are neither written nor read by anyone.)
 #include <atomic>
 #include <mutex>
 
@@ -22,7 +23,6 @@ namespace {
 
 static __device__ __align__(256) unsigned char g_static_workspace[APPROXIFER_STATIC_WORKSPACE_BYTES];
 
-constexpr int kMaxDevices = 64;
 std::mutex g_setup_mutex;
 unsigned char* g_workspace_ptr[kMaxDevices] = {};  // device address of g_static_workspace, per device
 
@@ -56,6 +56,7 @@ extern "C" int approxifer_encode_host_static(const approxifer_params* params, in
                                              float* hXt, void* cuda_stream) {
   if (params == nullptr) return APPROXIFER_E_NULL;
   if (params->K < 1 || params->K > APPROXIFER_MAX_K || params->W < 2 || params->W > APPROXIFER_MAX_W) return APPROXIFER_E_RANGE;
+  if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS)) return APPROXIFER_E_PARAM;
   if (G < 0 || D < 1 || D > (int64_t(1) << 31)) return APPROXIFER_E_RANGE;
   if (G == 0) return APPROXIFER_OK;
   if (hX == nullptr || hXt == nullptr) return APPROXIFER_E_NULL;
@@ -63,10 +64,11 @@ extern "C" int approxifer_encode_host_static(const approxifer_params* params, in
   // staging layout: [G][K][Dp] queries, then (256-byte aligned) [G][W][Dp] coded queries; Dp = D rounded up to
   // a multiple of 4 so that every row starts on a 16-byte boundary
   const int64_t Dp = (D + 3) & ~int64_t(3);
-  const unsigned long long in_bytes = (unsigned long long)G * K * Dp * 4, out_bytes = (unsigned long long)G * W * Dp * 4;
-  if (in_bytes > APPROXIFER_STATIC_WORKSPACE_BYTES || out_bytes > APPROXIFER_STATIC_WORKSPACE_BYTES ||
-      align256((size_t)in_bytes) + out_bytes > APPROXIFER_STATIC_WORKSPACE_BYTES)
+  // bound G by a division first, so that none of the products below can wrap (Dp <= 2^31 + 3, K + W <= 64)
+  if ((unsigned long long)G > APPROXIFER_STATIC_WORKSPACE_BYTES / (4ull * (unsigned long long)Dp * (unsigned long long)(K + W)))
     return APPROXIFER_E_TOO_LARGE;
+  const unsigned long long in_bytes = (unsigned long long)G * K * Dp * 4, out_bytes = (unsigned long long)G * W * Dp * 4;
+  if (align256((size_t)in_bytes) + out_bytes > APPROXIFER_STATIC_WORKSPACE_BYTES) return APPROXIFER_E_TOO_LARGE;
 
   unsigned char* base = nullptr;
   if (static_workspace(&base) != cudaSuccess) return APPROXIFER_E_CUDA;

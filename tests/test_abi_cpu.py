@@ -80,6 +80,50 @@ def test_decode_and_locate_argument_errors():
         assert lib.approxifer_locate(ctypes.byref(q), 0, 10, None, W * 10, 10, None, None, None, None, None) == want
 
 
+def test_flags_each_entry_point_ignores_or_rejects():
+    """One params struct serves the whole pipeline: the decoder's sign flag and the locator's homogeneous flag
+    are accepted (and ignored) by the entry points they do not concern; undefined bits are rejected everywhere."""
+    lib = ap.load()
+    both = binding.SIGN_WORKER_INDEX | binding.LOCATE_HOMOGENEOUS
+    q = ap.make_params(8, 24, 2, both)
+    bad = ap.make_params(8, 24, 2, 4)
+    assert lib.approxifer_encode(ctypes.byref(q), 0, 8, None, 64, 8, None, 192, 8, None) == binding.OK
+    assert lib.approxifer_encode(ctypes.byref(bad), 0, 8, None, 64, 8, None, 192, 8, None) == binding.E_PARAM
+    assert lib.approxifer_decode(ctypes.byref(q), 0, 10, None, 240, 10, None, None, 80, 10, None, None, None) == binding.OK
+    assert lib.approxifer_decode(ctypes.byref(bad), 0, 10, None, 240, 10, None, None, 80, 10, None, None, None) == binding.E_PARAM
+    assert lib.approxifer_locate(ctypes.byref(q), 0, 10, None, 240, 10, None, None, None, None, None) == binding.OK
+    assert lib.approxifer_locate(ctypes.byref(bad), 0, 10, None, 240, 10, None, None, None, None, None) == binding.E_PARAM
+    assert lib.approxifer_decode_rational(ctypes.byref(q), 0, 10, None, 240, 10, None, None, 80, 10, None, None) == binding.OK
+    assert lib.approxifer_decode_rational(ctypes.byref(bad), 0, 10, None, 240, 10, None, None, 80, 10, None, None) == binding.E_PARAM
+    assert lib.approxifer_encode_host_static(ctypes.byref(q), 0, 8, None, None, None) == binding.OK
+    assert lib.approxifer_encode_host_static(ctypes.byref(bad), 0, 8, None, None, None) == binding.E_PARAM
+
+
+def test_debug_entry_points_validate_their_tuning_on_the_host():
+    lib = ap.load()
+    p = ap.make_params(8, 12)
+    for (fields, want) in [((0, 0, 0, 0, 0), binding.OK), ((1, 0, 0, 0, 0), binding.OK), ((2, 0, 0, 0, 0), binding.E_PARAM),
+                           ((0, 1, 0, 0, 0), binding.E_PARAM), ((0, 0, -1, 0, 0), binding.E_PARAM), ((0, 0, 0, 48, 0), binding.E_PARAM),
+                           ((0, 0, 0, 0, 3), binding.E_PARAM), ((0, 4, 2, 256, 2), binding.OK)]:
+        t = binding.approxifer_decode_tuning(*fields)
+        rc = lib.approxifer_debug_decode(ctypes.byref(p), 0, 64, None, 768, 64, None, None, 512, 64, None, None, ctypes.byref(t), None)
+        assert rc == want, fields
+    assert lib.approxifer_debug_decode(ctypes.byref(p), 0, 64, None, 768, 64, None, None, 512, 64, None, None, None, None) == binding.OK
+    q = ap.make_params(8, 24, 2)
+    assert lib.approxifer_debug_locate(ctypes.byref(q), 0, 10, None, 240, 10, None, None, None, None, 1, None) == binding.OK
+    q = ap.make_params(8, 19, 2)
+    assert lib.approxifer_debug_locate(ctypes.byref(q), 0, 10, None, 240, 10, None, None, None, None, 1, None) == binding.E_PARAM
+
+
+def test_static_workspace_size_check_cannot_wrap():
+    """Group counts whose byte count overflows 64 bits are refused as too large before anything is enqueued."""
+    lib = ap.load()
+    p = ap.make_params(8, 12)
+    for G in (1 << 57, 1 << 60, (1 << 63) - 1):
+        assert lib.approxifer_encode_host_static(ctypes.byref(p), G, 3072, 1, 1, None) == binding.E_TOO_LARGE
+    assert lib.approxifer_encode_host_static(ctypes.byref(p), 1, 1 << 31, 1, 1, None) == binding.E_TOO_LARGE
+
+
 def test_binding_refuses_cpu_tensors():
     import torch
 

@@ -57,6 +57,13 @@ def test_decode_host_equals_device_entry_point(K, W, G, C, ws_mb, ns):
     ref = ap.approxifer_decode(p, hYt.to(dev()), hmask.to(dev()), n_used=n_used, status=status).cpu()
     assert torch.equal(hYh, ref)
     assert torch.equal(hn, n_used.cpu()) and torch.equal(hst, status.cpu())
+    # and against the fp64 checker, per group, at the decoder's tolerance
+    want, n_ref, st_ref = oracle.decode(K, W, hYt.numpy(), mask)
+    err = np.abs(hYh.numpy().astype(np.float64) - want).reshape(G, -1).max(axis=1)
+    scale = np.abs(want).reshape(G, -1).max(axis=1)
+    assert np.all(err <= 1e-4 * np.maximum(scale, 1e-30) + (scale == 0) * 0.0), float((err / np.maximum(scale, 1e-30)).max())
+    np.testing.assert_array_equal(hn.numpy(), n_ref)
+    np.testing.assert_array_equal(hst.numpy().view(np.uint32), st_ref)
 
 
 def test_locate_host_equals_device_entry_point():

@@ -274,17 +274,18 @@ def linear_case(K, W, E, S, G, C, seed, softmax=False, sigma=10.0, d_in=16):
     return torch.from_numpy(Y), mask, truth
 
 
-def run_locate(K, W, E, Yt, mask):
+def run_locate(K, W, E, Yt, mask, force_warp_kernel=False):
     G = Yt.shape[0]
     status = torch.empty(G, dtype=torch.int32, device=dev())
-    adv, trusted = ap.approxifer_locate(ap.make_params(K, W, E), Yt.to(dev()), ap.mask_tensor(mask), status=status)
+    adv, trusted = ap.approxifer_locate(ap.make_params(K, W, E), Yt.to(dev()), ap.mask_tensor(mask), status=status,
+                                        force_warp_kernel=force_warp_kernel)
     torch.cuda.synchronize()
     return adv.cpu().numpy(), trusted.cpu().numpy().view(np.uint32), status.cpu().numpy().view(np.uint32)
 
 
-def compare_locate(K, W, E, Yt, mask, allow_fragile=False):
+def compare_locate(K, W, E, Yt, mask, allow_fragile=False, force_warp_kernel=False):
     ref = oracle.locate(K, W, E, Yt.numpy(), mask)
-    adv, trusted, status = run_locate(K, W, E, Yt, mask)
+    adv, trusted, status = run_locate(K, W, E, Yt, mask, force_warp_kernel=force_warp_kernel)
     solid = (ref["min_gap"] > 1.0 + 1e-6) & (ref["vote_margin"] > 0) & ((ref["status"] & oracle.ST_ORACLE_RANK_DEFICIENT) == 0)
     solid |= (ref["status"] & oracle.ST_LOCATE_UNDERDETERMINED) != 0
     if not allow_fragile:
@@ -386,33 +387,30 @@ STAGED_SHAPES = [
                                                         (0, 0, 256, 2), (2, 1, 256, 0), (0, 0, 128, 0), (0, 0, 0, 1), (0, 0, 0, 2), (0, 0, 32, 2),
                                                         (3, 0, 32, 0), (0, 0, 16, 2)])
 def test_staged_decoder_matches_oracle_in_every_configuration(stages, ctas, cols, split):
-    try:
-        ap.debug_decode_config(stages, ctas, 0, cols, split)
-        for (K, W, G, C, flags) in STAGED_SHAPES:
-            rng = np.random.default_rng(C + K)
-            g = torch.Generator().manual_seed(C)
-            Yt = torch.randn((G, W, C), generator=g)
-            if flags == 0:
-                mask = random_masks(W, G, rng, min_present=0)
-                mask[0], mask[1], mask[2] = 2**W - 1, 0, 1 << (W - 1)
-            else:
-                mask = np.full(G, 2**W - 1, dtype=np.uint32)
-                mask[::3] = (2**W - 1) & ~1
-            dirty = Yt.clone()
-            for gi in range(G):
-                for i in range(W):
-                    if not (int(mask[gi]) >> i) & 1:
-                        dirty[gi, i] = float("nan")  # absent rows must never be used
-            n_used = torch.empty(G, dtype=torch.int32, device=dev())
-            status = torch.empty(G, dtype=torch.int32, device=dev())
-            out = torch.full((G, K, C + 4), CANARY, device=dev())
-            Yh = ap.approxifer_decode(ap.make_params(K, W, 0, flags), dirty.to(dev()), ap.mask_tensor(mask), out[:, :, :C],
-                                      n_used=n_used, status=status)
-            check_decode(K, W, Yt, mask, Yh, n_used, status, flags)
-            assert bool((out[:, :, C:] == CANARY).all())
-        assert ap.device_wait_timeouts() == 0
-    finally:
-        ap.debug_decode_config(0, 0, 0)
+    tuning = ap.decode_tuning(0, stages, ctas, cols, split)
+    for (K, W, G, C, flags) in STAGED_SHAPES:
+        rng = np.random.default_rng(C + K)
+        g = torch.Generator().manual_seed(C)
+        Yt = torch.randn((G, W, C), generator=g)
+        if flags == 0:
+            mask = random_masks(W, G, rng, min_present=0)
+            mask[0], mask[1], mask[2] = 2**W - 1, 0, 1 << (W - 1)
+        else:
+            mask = np.full(G, 2**W - 1, dtype=np.uint32)
+            mask[::3] = (2**W - 1) & ~1
+        dirty = Yt.clone()
+        for gi in range(G):
+            for i in range(W):
+                if not (int(mask[gi]) >> i) & 1:
+                    dirty[gi, i] = float("nan")  # absent rows must never be used
+        n_used = torch.empty(G, dtype=torch.int32, device=dev())
+        status = torch.empty(G, dtype=torch.int32, device=dev())
+        out = torch.full((G, K, C + 4), CANARY, device=dev())
+        Yh = ap.approxifer_decode(ap.make_params(K, W, 0, flags), dirty.to(dev()), ap.mask_tensor(mask), out[:, :, :C],
+                                  n_used=n_used, status=status, tuning=tuning)
+        check_decode(K, W, Yt, mask, Yh, n_used, status, flags)
+        assert bool((out[:, :, C:] == CANARY).all())
+    assert ap.device_wait_timeouts() == 0
 
 
 def test_staged_and_register_decoders_agree_bitwise_on_sums_order():
@@ -424,11 +422,7 @@ def test_staged_and_register_decoders_agree_bitwise_on_sums_order():
     mask = ap.mask_tensor(random_masks(W, G, rng, min_present=1))
     p = ap.make_params(K, W)
     a = ap.approxifer_decode(p, Yt, mask)
-    try:
-        ap.debug_decode_config(0, 0, 1)
-        b = ap.approxifer_decode(p, Yt, mask)
-    finally:
-        ap.debug_decode_config(0, 0, 0)
+    b = ap.approxifer_decode(p, Yt, mask, tuning=ap.decode_tuning(kernel=1))
     assert torch.equal(a, b)
 
 
@@ -460,11 +454,7 @@ def test_short_payload_decoder_against_oracle_and_register_decoder(K, W, C, G):
         if flags == 0:  # (the literal sign has poles: on arbitrary masks a denominator can vanish, see pin P9)
             check_decode(K, W, Yt, mask, Yh, n_used, status, flags)
         assert bool((guard[:32] == CANARY).all()) and bool((guard[32 + G * K * C:] == CANARY).all())
-        try:
-            ap.debug_decode_config(0, 0, 1)
-            ref = ap.approxifer_decode(p, dirty.to(dev()), ap.mask_tensor(mask))
-        finally:
-            ap.debug_decode_config(0, 0, 0)
+        ref = ap.approxifer_decode(p, dirty.to(dev()), ap.mask_tensor(mask), tuning=ap.decode_tuning(kernel=1))
         assert torch.equal(Yh.contiguous().view(torch.int32), ref.view(torch.int32))  # bit patterns: inf/NaN included
 
 
@@ -496,11 +486,7 @@ def test_both_locator_kernels_return_the_same_sets(K, E, S, W, C):
     Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=K + 7 * E + C)
     mask[5] = (1 << (2 * (K + E) - 1)) - 1  # one worker short: nothing to locate
     ref, adv_rows, _ = compare_locate(K, W, E, Yt, mask)
-    try:
-        ap.debug_locate_config(1)
-        ref2, adv_warp, _ = compare_locate(K, W, E, Yt, mask)
-    finally:
-        ap.debug_locate_config(0)
+    ref2, adv_warp, _ = compare_locate(K, W, E, Yt, mask, force_warp_kernel=True)
     np.testing.assert_array_equal(adv_rows, adv_warp)
     assert adv_rows[5, 0] == -1
 
