@@ -278,12 +278,16 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
  * Decoding", steps 1 and 2, exactly as in the two entry points they shadow).
  *
  * `tuning` (HOST pointer, read during the call; NULL = all automatic), every field 0 = automatic:
- *   kernel       1: route the call through the per-column register-staged kernel whatever the shape
+ *   kernel       1: route the call through the per-column register-staged kernel whatever the shape; 2, 3, 4: prefer
+ *                the thread-per-(query, chunk) kernel, the bulk-copy staged kernel, the packed-groups kernel where
+ *                that kernel takes the shape (else the automatic choice among the remaining ones)
  *   stages       bulk-copy staged kernel (rows of >= 64 floats on the 128-bit path): upper bound >= 2 on the ring depth
  *   ctas_per_sm  ... upper bound on resident CTAs per SM
  *   cols         ... 16, 32 (split 2 only), 64, 128 or 256 16-byte columns per work item (256 needs split 1 or 2
  *                and a ring that fits in shared memory, else 128 is used)
  *   split        ... 1 (K <= 16, 256 columns), 2 or 4 thread groups sharing the K queries of a column
+ *   For the packed-groups kernel (dense buffers, even C <= 62) `stages` = 2..4 sets each warp's ring depth,
+ *   `ctas_per_sm` bounds the warps per CTA and `cols` (any positive value) the groups per work item.
  * APPROXIFER_E_PARAM for any other value.
  *
  * force_warp_kernel != 0 routes the locate through the warp-per-group kernel, which otherwise serves only

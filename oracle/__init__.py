@@ -19,6 +19,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "approxifer_oracle.c")
+_SRC_BF16 = os.path.join(_HERE, "bf16_oracle.c")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
 ST_NO_WORKERS = 1
@@ -32,11 +33,11 @@ FLAG_SIGN_WORKER_INDEX = 1
 
 def build(force: bool = False) -> str:
     """Compile the oracle if the shared object is missing or older than the source."""
-    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_BF16))
     if force or stale:
         tmp = _LIB + ".tmp.%d" % os.getpid()
         subprocess.check_call(
-            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, _SRC_BF16, "-lm"]
         )
         os.replace(tmp, _LIB)
     return _LIB
@@ -71,6 +72,13 @@ def _load():
     lib.oracle_locate_class.restype = c_int
     lib.oracle_locate.argtypes = [c_int, c_int, c_int, c_int64, c_int64, pf, c_int64, c_int64, pu,
                                   pi, pu, pu, pd, pi]
+    pu16 = POINTER(ctypes.c_uint16)
+    lib.oracle_bf16_to_double.argtypes = [ctypes.c_uint16]
+    lib.oracle_bf16_to_double.restype = c_double
+    lib.oracle_double_to_bf16.argtypes = [c_double]
+    lib.oracle_double_to_bf16.restype = ctypes.c_uint16
+    lib.oracle_bf16_widen.argtypes = [c_int64, pu16, pf]
+    lib.oracle_bf16_round.argtypes = [c_int64, pd, pu16]
     _lib = lib
     return lib
 
@@ -209,3 +217,41 @@ def locate(K: int, W: int, E: int, Yt, mask):
     _load().oracle_locate(K, W, E, G, C, _p(Yt, c_float), gs, rs, _p(mask, c_uint32), _p(adv, c_int32),
                           _p(trusted, c_uint32), _p(status, c_uint32), _p(gap, c_double), _p(margin, c_int32))
     return dict(adv=adv, trusted=trusted, status=status, min_gap=gap, vote_margin=margin)
+
+
+# ---- bfloat16 storage (bf16_oracle.c): exact widening, the fp64 formulas above, one rounding to nearest-even ----
+
+def bf16_to_double(bits: int) -> float:
+    return float(_load().oracle_bf16_to_double(int(bits) & 0xFFFF))
+
+
+def double_to_bf16(x: float) -> int:
+    return int(_load().oracle_double_to_bf16(float(x)))
+
+
+def bf16_widen(bits) -> np.ndarray:
+    """uint16 bfloat16 bit patterns -> the float32 array of the same values (exact)."""
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    out = np.empty(b.shape, dtype=np.float32)
+    _load().oracle_bf16_widen(b.size, _p(b, ctypes.c_uint16), _p(out, c_float))
+    return out
+
+
+def bf16_round(x) -> np.ndarray:
+    """float64 array -> uint16 bit patterns of the nearest bfloat16 (ties to even)."""
+    a = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.empty(a.shape, dtype=np.uint16)
+    _load().oracle_bf16_round(a.size, _p(a, c_double), _p(out, ctypes.c_uint16))
+    return out
+
+
+def encode_bf16(K: int, W: int, X_bits):
+    """Encoder on bfloat16 queries [G][K][D] (uint16 bit patterns): (exact fp64 coded queries, their bfloat16 roundings)."""
+    exact = encode(K, W, bf16_widen(X_bits))
+    return exact, bf16_round(exact)
+
+
+def decode_bf16(K: int, W: int, Yt_bits, mask, flags: int = 0):
+    """Decoder on bfloat16 predictions [G][W][C]: (exact fp64 result, its bfloat16 rounding, n_used, status)."""
+    exact, n_used, status = decode(K, W, bf16_widen(Yt_bits), mask, flags)
+    return exact, bf16_round(exact), n_used, status

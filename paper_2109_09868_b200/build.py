@@ -20,7 +20,7 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 OBJDIR = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libapproxifer.so")
 
-SOURCES = ["api.cu", "tables.cpp", "encode.cu", "decode.cu", "decode_small.cu", "decode_staged.cu", "locate.cu", "locate_rows.cu", "locate_rows_n8.cu", "locate_rows_n16.cu", "locate_rows_n24.cu", "locate_rows_n32.cu", "host_api.cu", "no_alloc.cu"]
+SOURCES = ["api.cu", "tables.cpp", "encode.cu", "decode.cu", "decode_small.cu", "decode_pack.cu", "decode_staged.cu", "locate.cu", "locate_rows.cu", "locate_rows_n8.cu", "locate_rows_n16.cu", "locate_rows_n24.cu", "locate_rows_n32.cu", "host_api.cu", "no_alloc.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 CFLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--expt-relaxed-constexpr"]
 

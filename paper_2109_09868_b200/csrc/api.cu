@@ -119,8 +119,8 @@ int approxifer_debug_decode(const approxifer_params* params, int64_t G, int64_t 
   DecodeTuning t{};
   if (tuning != nullptr) {
     const int cols = tuning->cols, split = tuning->split;
-    if (tuning->kernel < 0 || tuning->kernel > 1 || tuning->stages < 0 || tuning->stages == 1 || tuning->ctas_per_sm < 0 ||
-        (cols != 0 && cols != 16 && cols != 32 && cols != 64 && cols != 128 && cols != 256) ||
+    if (tuning->kernel < 0 || tuning->kernel > 4 || tuning->stages < 0 || tuning->stages == 1 || tuning->ctas_per_sm < 0 ||
+        cols < 0 || (tuning->kernel != 4 && cols != 0 && cols != 16 && cols != 32 && cols != 64 && cols != 128 && cols != 256) ||
         (split != 0 && split != 1 && split != 2 && split != 4))
       return APPROXIFER_E_PARAM;
     t.kernel = tuning->kernel, t.stages = tuning->stages, t.ctas_per_sm = tuning->ctas_per_sm, t.cols = cols, t.split = split;
@@ -187,9 +187,9 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
 }
 
 int64_t approxifer_device_wait_timeouts(void) {
-  unsigned int n = 0;
-  if (read_decode_wait_timeouts(&n) != cudaSuccess) return -1;
-  return (int64_t)n;
+  unsigned int n = 0, m = 0;
+  if (read_decode_wait_timeouts(&n) != cudaSuccess || read_pack_wait_timeouts(&m) != cudaSuccess) return -1;
+  return (int64_t)n + (int64_t)m;
 }
 
 const char* approxifer_strerror(int code) {

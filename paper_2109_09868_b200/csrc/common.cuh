@@ -28,7 +28,8 @@ struct EncodeArgs {
 
 // Test / tuning choices of one decode call (all zero = automatic); see approxifer_debug_decode.
 struct DecodeTuning {
-  int32_t kernel = 0;       // 0 automatic, 1 the per-column register-staged kernel
+  int32_t kernel = 0;       // 0 automatic; 1 per-column register-staged, 2 thread-per-(query, chunk), 3 bulk-copy
+                            // staged, 4 packed-groups kernel (2..4: only where the kernel takes the shape)
   int32_t stages = 0;       // bulk-copy staged kernel: upper bound on the ring depth
   int32_t ctas_per_sm = 0;  // ... upper bound on resident CTAs per SM
   int32_t cols = 0;         // ... 16-byte columns per work item
@@ -75,6 +76,11 @@ cudaError_t launch_debug_weights(int K, int W, uint32_t flags, uint32_t mask, in
 bool decode_staged_eligible(const DecodeArgs& a);
 cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream);
 cudaError_t read_decode_wait_timeouts(unsigned int* out);
+
+// Short- and medium-payload decoder for dense buffers (groups packed into work items); see decode_pack.cu.
+bool decode_pack_eligible(const DecodeArgs& a);
+cudaError_t launch_decode_pack(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream);
+cudaError_t read_pack_wait_timeouts(unsigned int* out);
 
 // Short-payload decoder (C <= 32, dense buffers); see decode_small.cu.
 bool decode_small_eligible(const DecodeArgs& a);

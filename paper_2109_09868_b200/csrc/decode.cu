@@ -228,6 +228,7 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
   const DecodeTables& tab = decode_tables(a.K, a.W);
   const bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&
                    a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  if (decode_pack_eligible(a)) return launch_decode_pack(a, tab, stream);
   if (decode_small_eligible(a)) return launch_decode_small(a, tab, stream);
   if (decode_staged_eligible(a)) return launch_decode_staged(a, tab, stream);
   if (vec) return dispatch_k<float4>(a, tab, stream);

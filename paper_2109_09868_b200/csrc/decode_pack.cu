@@ -1,0 +1,425 @@
+// ApproxIFER decoder for short payloads in dense buffers (Section 3, "Decoding", step 2): predictions of an even
+// number of classes up to 62 -- the paper's own workloads have C = 10 -- stored back to back ([G][W][C] in,
+// [G][K][C] out).
+//
+// Same arithmetic as decode_kernel, term by term and rounding by rounding (barycentric numerator and
+// denominator over the present workers in ascending order, one reciprocal per query), different data movement
+// and work split:
+//
+//  * Every WARP is a pipeline of its own.  A warp's work item is a block of GW consecutive groups (a few KB,
+//    one contiguous range: rows this short are shorter than a DRAM burst, so the absent workers' rows come
+//    along and are simply never used).  Lane 0 brings items into the warp's private shared-memory ring with
+//    bulk asynchronous copies, S-1 items ahead of the one being reduced, completion counted on one mbarrier
+//    per slot; a slot is refilled by the warp that has just finished reading it, so there are no "empty"
+//    barriers, no producer warp and no CTA-wide barrier in the main loop.  With a dozen such warps per SM
+//    there are always tens of KB of loads in flight and always some warp with arithmetic to do.
+//  * Lane = (group of the item, tile of two queries, word lane).  A thread forms two queries for NW words
+//    (pairs of adjacent classes): every payload word it loads from shared memory feeds two packed
+//    multiply-adds (fma.rn.f32x2: both halves ordinary round-to-nearest fp32 FMAs), and the signed weights
+//    and denominators of its queries are formed once per worker.  All lanes step through the workers
+//    0 .. W-1 together and skip (by predicate) those absent from their group's mask, so a warp reads one
+//    table row and one row position at a time; a worker's rank (its sign) is a running population count.
+//  * Results are collected in the ring slot they were computed from (its predictions are no longer needed, and
+//    K rows never take more room than W) and streamed out by the whole warp with 128-bit stores, again one
+//    contiguous range.  (A bulk copy out of shared memory frees its source only after
+//    several microseconds; waiting for that dominated every variant that used one.)
+//
+// Every wait is bounded.  Every bulk copy targets, or reads, the issuing CTA's own shared memory.
+#include "common.cuh"
+
+namespace approxifer {
+
+__device__ unsigned int g_pack_wait_timeouts = 0;  // bounded waits that gave up (never, in a correct run)
+
+namespace {
+
+constexpr int kPackMaxWarps = 24;
+// warps per CTA by words per lane: short rows leave room for 24 warps of 80 registers, longer ones get 16 of 128
+__host__ __device__ constexpr int pack_max_warps(int nw) { return nw <= 5 ? kPackMaxWarps : 16; }
+constexpr int kPackMaxStages = 4;
+constexpr int kPackMaxNW = 10;  // words (float2) per thread and row
+constexpr int kPackMaxC = 62;
+constexpr uint32_t kPackWaitLimit = 1u << 22;
+constexpr unsigned kFullMask = 0xffffffffu;
+
+__device__ __forceinline__ uint32_t p_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void p_mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void p_fence_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void p_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool p_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// global -> this CTA's shared memory; src, dst and bytes are multiples of 16
+__device__ __forceinline__ void p_bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ uint64_t p_ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t p_dup(float v) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %1};" : "=l"(d) : "r"(__float_as_uint(v)));
+  return d;
+}
+
+struct PackPlan {
+  int32_t gw;         // groups per warp item
+  int32_t nch;        // lanes sharing the words of one (group, query tile)
+  int32_t jt;         // query tiles per group = ceil(K / 2)
+  int32_t stages;     // ring depth per warp
+  int32_t warps;      // warps per CTA
+  int32_t in_bytes;   // one ring slot (gw * W * C floats, padded to 128 B)
+  int32_t table_bytes;
+  int64_t n_items;
+};
+
+__device__ __forceinline__ float p_lo(uint64_t v) { return __uint_as_float((uint32_t)v); }
+__device__ __forceinline__ float p_hi(uint64_t v) { return __uint_as_float((uint32_t)(v >> 32)); }
+
+// Shared memory: wtab[2][W][KP] (8 bytes each) | coin[32] | per warp: full[S] mbarriers (64 B) | S ring slots.
+// wtab[sg][i][j] = (w, w) with w = (-1)^sg / (alpha_j - beta_i): the signed weight, already duplicated for the
+// packed multiply-add (the sign flip is exact, so (s rg) y rounds like rg (s y)).
+// SIMPLE: one lane owns all the words of its rows (nch == 1, NW == C/2), so every offset is a compile-time constant.
+template <int NW, bool SIMPLE>
+__global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
+    decode_pack_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ DecodeTables tab,
+                       const __grid_constant__ PackPlan plan) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int W = a.W, K = a.K, C = (int)a.C, S = plan.stages, GW = plan.gw;
+  const int KP = (K + 1) & ~1;
+  uint64_t* wtab = reinterpret_cast<uint64_t*>(smem_raw);           // [2][W][KP], 0 beyond K
+  int* coins = reinterpret_cast<int*>(smem_raw + 2 * W * KP * 8);  // [32]
+  const uint32_t per_warp = 64u + (uint32_t)S * (uint32_t)plan.in_bytes;
+  unsigned char* mine = smem_raw + plan.table_bytes + (size_t)warp * per_warp;
+  uint64_t* full = reinterpret_cast<uint64_t*>(mine);
+  unsigned char* slots = mine + 64;
+  const uint32_t wb = worker_bits(W);
+  const uint32_t group_bytes = (uint32_t)(W * C * 4);
+  const uint32_t row_bytes = (uint32_t)(C * 4);
+
+  for (int idx = tid; idx < 2 * W * KP; idx += blockDim.x) {
+    const int sg = idx / (W * KP), rem = idx - sg * (W * KP);
+    const int i = rem / KP, j = rem - i * KP;
+    const float w = (j < K) ? tab.rg[i * K + j] : 0.f;
+    wtab[idx] = p_dup(sg ? -w : w);
+  }
+  if (tid < 32) coins[tid] = (tab.any_coin && tid < K) ? (int)tab.coin[tid] : -1;
+  if (lane == 0) {
+    for (int s = 0; s < S; ++s) p_mbar_init(p_smem_u32(full + s), 1);
+    p_fence_init();
+  }
+  __syncthreads();
+
+  // items are dealt to the warps of the whole grid round-robin: neighbouring warps work on neighbouring memory
+  const int64_t first = (int64_t)blockIdx.x * plan.warps + warp, stride = (int64_t)gridDim.x * plan.warps;
+  const int64_t my_items = first < plan.n_items ? (plan.n_items - first + stride - 1) / stride : 0;
+
+  // lane = (group s of the item, query tile jt, word lane ch)
+  const int nch = SIMPLE ? 1 : plan.nch, JT = plan.jt;
+  const int sj = lane / nch, ch = lane - sj * nch;
+  const int s = sj / JT, jt = sj - s * JT;
+  const int j0 = jt * 2;
+  const int Cw = C >> 1;
+  const bool exact = SIMPLE || NW * nch == Cw;  // no lane has a word beyond the end of the row
+  const bool literal = (a.flags & kFlagSignWorkerIndex) != 0;
+  const uint32_t y_off = (uint32_t)s * group_bytes + (uint32_t)ch * 8u;
+  const uint32_t u_step = (uint32_t)nch * 8u;
+  const int c0 = (j0 < K) ? coins[j0] : -1, c1 = (j0 + 1 < K) ? coins[j0 + 1] : -1;
+  const uint32_t sign_step = (uint32_t)(W * KP) * 8u;  // bytes between the two signs of the table
+  const unsigned char* wrow0 = reinterpret_cast<const unsigned char*>(wtab) + (uint32_t)j0 * 8u;
+
+  // lane 0: start the copy of the item whose first group is g0 into ring slot `slot`.  A ragged last item may end
+  // on an 8-byte boundary: the copy takes the whole 16-byte columns and the last two floats go by hand.
+  auto issue = [&](int64_t g0, int slot) {
+    const int ng = (int)min((int64_t)GW, a.G - g0);
+    const uint32_t bytes = (uint32_t)ng * group_bytes, bytes16 = bytes & ~15u;
+    const unsigned char* src = reinterpret_cast<const unsigned char*>(a.Yt + g0 * (int64_t)(W * C));
+    unsigned char* dst = slots + (size_t)slot * plan.in_bytes;
+    const uint32_t bar = p_smem_u32(full + slot);
+    if (bytes16 != bytes) *reinterpret_cast<float2*>(dst + bytes16) = *reinterpret_cast<const float2*>(src + bytes16);
+    p_arrive_expect_tx(bar, bytes16);  // (release: the two floats above are visible to whoever sees the phase complete)
+    if (bytes16) p_bulk_g2s(p_smem_u32(dst), src, bytes16, bar);
+  };
+  // this lane's group's mask in the item whose first group is g0 (0 beyond the end)
+  auto fetch_mask = [&](int64_t g0) -> uint32_t {
+    const int64_t g = g0 + s;
+    return (s < GW && g < a.G) ? (a.mask[g] & wb) : 0u;
+  };
+
+  // prologue: S-1 items in flight, their masks in registers (mq0 belongs to the item about to be reduced)
+  const int64_t g_first = first * GW, g_stride = stride * GW;
+  const int64_t g_end = g_first + my_items * g_stride;  // first group of the item after this warp's last
+  uint32_t mq0 = 0u, mq1 = 0u, mq2 = 0u;
+  if (S > 1 && 0 < my_items) mq0 = fetch_mask(g_first);
+  if (S > 2 && 1 < my_items) mq1 = fetch_mask(g_first + g_stride);
+  if (S > 3 && 2 < my_items) mq2 = fetch_mask(g_first + 2 * g_stride);
+  if (lane == 0)
+    for (int d = 0; d < S - 1 && d < my_items; ++d) issue(g_first + d * g_stride, d);
+
+  int64_t g0 = g_first;                             // first group of the item being reduced
+  int64_t g_ahead = g_first + (S - 1) * g_stride;   // ... of the item started in the same iteration
+  int slot = 0, slot_ahead = S - 1;                 // their ring slots
+  uint32_t parity = 0;
+  int64_t failed_g0 = -1;
+  for (; g0 < g_end; g0 += g_stride, g_ahead += g_stride) {
+    const int ng = (int)min((int64_t)GW, a.G - g0);
+    // the slot that the previous item occupied is free (its results were copied out of it before the __syncwarp
+    // that ended the previous iteration): refill it with the item S-1 ahead, and fetch that item's mask
+    uint32_t m_new = 0u;
+    if (g_ahead < g_end) {
+      m_new = fetch_mask(g_ahead);
+      if (lane == 0) issue(g_ahead, slot_ahead);
+    }
+    // wait for this item's bytes (bounded)
+    {
+      const uint32_t addr = p_smem_u32(full + slot);
+      bool ok = false;
+      for (uint32_t it = 0; it < kPackWaitLimit && !ok; ++it) ok = p_try_wait(addr, parity);
+      if (!__all_sync(kFullMask, ok)) {
+        if (lane == 0) atomicAdd(&g_pack_wait_timeouts, 1u);
+        failed_g0 = g0;
+        break;
+      }
+    }
+    const uint32_t mask = mq0;
+    const unsigned char* yg = slots + (size_t)slot * plan.in_bytes + y_off;
+    uint64_t acc0[NW], acc1[NW];  // numerators of this lane's two queries, a pair of classes per word
+    float inv0 = 0.f, inv1 = 0.f;
+    bool pin0 = false, pin1 = false;
+    int n = 0;
+    if (s < ng) {
+#pragma unroll
+      for (int u = 0; u < NW; ++u) acc0[u] = acc1[u] = 0ull;
+      float den0 = 0.f, den1 = 0.f;
+      uint32_t r = 0;  // present workers so far = rank of the next one
+      const unsigned char* yr = yg;
+      const unsigned char* wr = wrow0;
+#pragma unroll(NW <= 7 ? 2 : 1)
+      for (int i = 0; i < W; ++i, yr += row_bytes, wr += KP * 8) {
+        uint64_t y[NW];
+#pragma unroll
+        for (int u = 0; u < NW; ++u) {  // (an absent worker's row may be loaded; it is only used under `present`)
+          if constexpr (SIMPLE) y[u] = reinterpret_cast<const uint64_t*>(yr)[u];
+          else y[u] = (exact || u * nch + ch < Cw) ? *reinterpret_cast<const uint64_t*>(yr + u * u_step) : 0ull;
+        }
+        if ((mask >> i) & 1u) {
+          // the signed, duplicated weights of this lane's two queries
+          const uint32_t odd = (literal ? (uint32_t)i : r) & 1u;
+          const ulonglong2 w2 = *reinterpret_cast<const ulonglong2*>(wr + odd * sign_step);
+          den0 = __fadd_rn(den0, p_lo(w2.x));
+          den1 = __fadd_rn(den1, p_lo(w2.y));
+#pragma unroll
+          for (int u = 0; u < NW; ++u) {
+            acc0[u] = p_ffma2(w2.x, y[u], acc0[u]);
+            acc1[u] = p_ffma2(w2.y, y[u], acc1[u]);
+          }
+          ++r;
+        }
+      }
+      n = (int)r;
+      // alpha_j == beta_i for a present worker i: the interpolant takes that worker's value
+      pin0 = c0 >= 0 && ((mask >> c0) & 1u), pin1 = c1 >= 0 && ((mask >> c1) & 1u);
+      inv0 = __frcp_rn(den0), inv1 = __frcp_rn(den1);
+      if (pin0 || pin1) {
+#pragma unroll
+        for (int u = 0; u < NW; ++u) {
+          if (exact || u * nch + ch < Cw) {
+            if (pin0) acc0[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c0 * row_bytes + u * u_step);
+            if (pin1) acc1[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c1 * row_bytes + u * u_step);
+          }
+        }
+      }
+    }
+    __syncwarp();  // every lane has finished reading the slot: the results take its place
+    unsigned char* ob = slots + (size_t)slot * plan.in_bytes;
+    if (s < ng) {
+      unsigned char* orow = ob + (size_t)(s * K + j0) * row_bytes + (size_t)ch * 8u;
+#pragma unroll
+      for (int u = 0; u < NW; ++u) {
+        if (exact || u * nch + ch < Cw) {
+          float2 v0 = pin0 ? make_float2(p_lo(acc0[u]), p_hi(acc0[u])) : make_float2(p_lo(acc0[u]) * inv0, p_hi(acc0[u]) * inv0);
+          float2 v1 = pin1 ? make_float2(p_lo(acc1[u]), p_hi(acc1[u])) : make_float2(p_lo(acc1[u]) * inv1, p_hi(acc1[u]) * inv1);
+          if (n == 0) v0 = v1 = make_float2(0.f, 0.f);
+          if (j0 < K) *reinterpret_cast<float2*>(orow + u * u_step) = v0;
+          if (j0 + 1 < K) *reinterpret_cast<float2*>(orow + row_bytes + u * u_step) = v1;
+        }
+      }
+      if (jt == 0 && ch == 0) {
+        if (a.n_used) a.n_used[g0 + s] = n;
+        if (a.status) a.status[g0 + s] = (n == 0 ? kStNoWorkers : 0u) | (n < K ? kStFewWorkers : 0u);
+      }
+    }
+    __syncwarp();  // all results are in place
+    {
+      // the item's results are one contiguous range: the warp streams it out in whole 16-byte columns (a ragged
+      // last item may end on an 8-byte boundary)
+      const uint32_t bytes = (uint32_t)ng * (uint32_t)(K * C * 4), n16 = bytes >> 4;
+      unsigned char* dst = reinterpret_cast<unsigned char*>(a.Yh + g0 * (int64_t)(K * C));
+      for (uint32_t q = lane; q < n16; q += 32)
+        st_stream(reinterpret_cast<float4*>(dst) + q, reinterpret_cast<const float4*>(ob)[q]);
+      if (lane == 0 && (bytes & 15u))
+        __stcs(reinterpret_cast<float2*>(dst + (n16 << 4)), *reinterpret_cast<const float2*>(ob + (n16 << 4)));
+    }
+    __syncwarp();  // the slot may be refilled
+    // masks move up the queue; the newly fetched one joins at position S-2
+    mq0 = mq1, mq1 = mq2;
+    if (S == 2) mq0 = m_new;
+    else if (S == 3) mq1 = m_new;
+    else mq2 = m_new;
+    slot_ahead = slot;
+    if (++slot == S) {
+      slot = 0;
+      parity ^= 1u;
+    }
+  }
+  if (lane == 0 && failed_g0 >= 0) {
+    // the copies of the failed item and of the S-1 after it have been started: they must land before the CTA's
+    // shared memory is given up (bounded)
+    for (int d = 0; d < S && failed_g0 + d * g_stride < g_end; ++d) {
+      const uint32_t addr = p_smem_u32(full + slot);
+      for (uint32_t it = 0; it < kPackWaitLimit; ++it)
+        if (p_try_wait(addr, parity)) break;
+      if (++slot == S) {
+        slot = 0;
+        parity ^= 1u;
+      }
+    }
+  }
+}
+
+struct PackChoice {
+  int nw = 0, nch = 0, jt = 0, gw = 0, stages = 0, warps = 0;
+  int in_bytes = 0, table_bytes = 0, smem = 0;
+};
+
+// How the words of a row are dealt to lanes: NW words per lane, nch lanes per (group, query tile).  Exact splits
+// are preferred (no predicated tail), then more words per lane.
+void choose_words(int Cw, int* nw, int* nch) {
+  int best_nw = 1, best_waste = 1 << 30;
+  for (int w = kPackMaxNW; w >= 1; --w) {
+    const int n = (Cw + w - 1) / w;
+    const int waste = n * w - Cw;
+    if (waste < best_waste && (w >= 4 || Cw < 4 || waste == 0)) best_nw = w, best_waste = waste;
+  }
+  *nw = best_nw;
+  *nch = (Cw + best_nw - 1) / best_nw;
+}
+
+bool plan_pack(const DecodeArgs& a, int smem_per_sm, PackChoice* out) {
+  PackChoice p;
+  const int K = a.K, W = a.W, C = (int)a.C;
+  if (C < 2 || C > kPackMaxC || (C & 1)) return false;
+  p.jt = (K + 1) / 2;
+  choose_words(C / 2, &p.nw, &p.nch);
+  const int lpg = p.jt * p.nch;  // lanes per group
+  if (lpg > 32) return false;
+  int gw = 32 / lpg;
+  if (a.tune.cols > 0 && a.tune.cols < gw) gw = a.tune.cols;  // (tuning: upper bound on the groups per item)
+  if ((int64_t)gw > a.G) gw = (int)a.G;
+  // every item, and its block of results, starts on a 16-byte boundary
+  while (gw >= 1 && (int64_t)gw < a.G && (((int64_t)gw * W * C) % 4 != 0 || ((int64_t)gw * K * C) % 4 != 0)) --gw;
+  if (gw < 1) return false;
+  p.gw = gw;
+  if (K > W) return false;  // (the results of an item are staged in the slot of its predictions)
+  p.in_bytes = (gw * W * C * 4 + 127) & ~127;
+  const int KP = (K + 1) & ~1;
+  p.table_bytes = (2 * W * KP * 8 + 128 + 127) & ~127;
+  const int budget = smem_per_sm - 1024 - p.table_bytes;
+  // Two slots per warp: one item in flight while one is reduced.  What hides the latency of the loads is the
+  // number of warps (each with an item in flight), not the depth of a warp's ring: measured, 22 warps with two
+  // slots beat 16 with three and 12 with four.
+  int stages = 2;
+  if (a.tune.stages >= 2 && a.tune.stages <= kPackMaxStages) stages = a.tune.stages;
+  const int per_warp = 64 + stages * p.in_bytes;
+  int warps = budget / per_warp;
+  if (warps > pack_max_warps(p.nw)) warps = pack_max_warps(p.nw);
+  if (a.tune.ctas_per_sm > 0 && a.tune.ctas_per_sm < warps) warps = a.tune.ctas_per_sm;  // (tuning: warps per CTA)
+  if (warps < 4) return false;
+  p.stages = stages;
+  p.warps = warps;
+  p.smem = p.table_bytes + warps * per_warp;
+  *out = p;
+  return true;
+}
+
+template <int NW, bool SIMPLE>
+cudaError_t launch_pack(const DecodeArgs& a, const DecodeTables& tab, const PackChoice& c, const DeviceInfo& di,
+                        cudaStream_t stream) {
+  PackPlan plan;
+  plan.gw = c.gw, plan.nch = c.nch, plan.jt = c.jt, plan.stages = c.stages, plan.warps = c.warps;
+  plan.in_bytes = c.in_bytes, plan.table_bytes = c.table_bytes;
+  plan.n_items = (a.G + c.gw - 1) / c.gw;
+  struct Tag {};
+  cudaError_t e = ensure_dynamic_smem<Tag>(decode_pack_kernel<NW, SIMPLE>, di.ordinal, c.smem);
+  if (e != cudaSuccess) return e;
+  int64_t grid = di.sms;
+  const int64_t need = (plan.n_items + c.warps - 1) / c.warps;
+  if (grid > need) grid = need;
+  decode_pack_kernel<NW, SIMPLE><<<(unsigned)grid, c.warps * 32, c.smem, stream>>>(a, tab, plan);
+  count_launch();
+  return cudaGetLastError();
+}
+
+template <int NW = 1>
+cudaError_t dispatch_nw(const DecodeArgs& a, const DecodeTables& tab, const PackChoice& c, const DeviceInfo& di,
+                        cudaStream_t stream) {
+  if constexpr (NW > kPackMaxNW) {
+    return cudaErrorInvalidValue;
+  } else {
+    if (c.nw == NW) {
+      if (c.nch == 1 && NW * 2 == a.C) return launch_pack<NW, true>(a, tab, c, di, stream);
+      return launch_pack<NW, false>(a, tab, c, di, stream);
+    }
+    return dispatch_nw<NW + 1>(a, tab, c, di, stream);
+  }
+}
+
+}  // namespace
+
+// Dense buffers (rows and groups back to back), 16-byte aligned, an even number of classes up to 62.
+bool decode_pack_eligible(const DecodeArgs& a) {
+  if (a.tune.kernel != 0 && a.tune.kernel != 4) return false;
+  if (a.y_rs != a.C || a.y_gs != (int64_t)a.W * a.C || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
+  if (!aligned16(a.Yt) || !aligned16(a.Yh)) return false;
+  const DeviceInfo* di = nullptr;
+  if (current_device_info(&di) != cudaSuccess) return false;
+  PackChoice c;
+  return plan_pack(a, di->smem_per_sm, &c);
+}
+
+cudaError_t read_pack_wait_timeouts(unsigned int* out) {
+  return cudaMemcpyFromSymbol(out, g_pack_wait_timeouts, sizeof(unsigned int));
+}
+
+cudaError_t launch_decode_pack(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream) {
+  const DeviceInfo* di = nullptr;
+  cudaError_t e = current_device_info(&di);
+  if (e != cudaSuccess) return e;
+  PackChoice c;
+  if (!plan_pack(a, di->smem_per_sm, &c)) return cudaErrorInvalidConfiguration;
+  return dispatch_nw<>(a, tab, c, *di, stream);
+}
+
+}  // namespace approxifer

@@ -219,7 +219,7 @@ cudaError_t dispatch_cp(const DecodeArgs& a, const DecodeTables& tab, const Chun
 // Dense buffers (rows and groups back to back), 16-byte aligned, a class count that cuts into chunks (see
 // plan_chunks), and room for at least one group per CTA.
 bool decode_small_eligible(const DecodeArgs& a) {
-  if (a.tune.kernel == 1) return false;
+  if (a.tune.kernel != 0 && a.tune.kernel != 2) return false;
   if (a.y_rs != a.C || a.y_gs != (int64_t)a.W * a.C || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
   if (!aligned16(a.Yt) || !aligned16(a.Yh)) return false;
   const ChunkPlan p = plan_chunks(a.C);

@@ -455,7 +455,7 @@ cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cu
 // C = 200 on, where they reach 2.1-3.8 TB/s; at C = 40-48 they are as fast or faster).  Narrower payloads, and
 // the (K, W) pairs in which some alpha_j equals some beta_i (the row-copy case), stay on the other kernels.
 bool decode_staged_eligible(const DecodeArgs& a) {
-  if (a.tune.kernel == 1) return false;
+  if (a.tune.kernel != 0 && a.tune.kernel != 3) return false;
   const bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&
                    a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
   if (!(vec && a.C >= kStagedMinC)) return false;

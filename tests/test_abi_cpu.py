@@ -102,7 +102,7 @@ def test_flags_each_entry_point_ignores_or_rejects():
 def test_debug_entry_points_validate_their_tuning_on_the_host():
     lib = ap.load()
     p = ap.make_params(8, 12)
-    for (fields, want) in [((0, 0, 0, 0, 0), binding.OK), ((1, 0, 0, 0, 0), binding.OK), ((2, 0, 0, 0, 0), binding.E_PARAM),
+    for (fields, want) in [((0, 0, 0, 0, 0), binding.OK), ((1, 0, 0, 0, 0), binding.OK), ((5, 0, 0, 0, 0), binding.E_PARAM), ((4, 0, 0, 7, 0), binding.OK),
                            ((0, 1, 0, 0, 0), binding.E_PARAM), ((0, 0, -1, 0, 0), binding.E_PARAM), ((0, 0, 0, 48, 0), binding.E_PARAM),
                            ((0, 0, 0, 0, 3), binding.E_PARAM), ((0, 4, 2, 256, 2), binding.OK)]:
         t = binding.approxifer_decode_tuning(*fields)

@@ -387,7 +387,7 @@ STAGED_SHAPES = [
                                                         (0, 0, 256, 2), (2, 1, 256, 0), (0, 0, 128, 0), (0, 0, 0, 1), (0, 0, 0, 2), (0, 0, 32, 2),
                                                         (3, 0, 32, 0), (0, 0, 16, 2)])
 def test_staged_decoder_matches_oracle_in_every_configuration(stages, ctas, cols, split):
-    tuning = ap.decode_tuning(0, stages, ctas, cols, split)
+    tuning = ap.decode_tuning(3, stages, ctas, cols, split)
     for (K, W, G, C, flags) in STAGED_SHAPES:
         rng = np.random.default_rng(C + K)
         g = torch.Generator().manual_seed(C)
@@ -450,12 +450,88 @@ def test_short_payload_decoder_against_oracle_and_register_decoder(K, W, C, G):
         status = torch.empty(G, dtype=torch.int32, device=dev())
         guard = torch.full((G * K * C + 64,), CANARY, device=dev())
         Yh = guard[32: 32 + G * K * C].view(G, K, C)
-        ap.approxifer_decode(p, dirty.to(dev()), ap.mask_tensor(mask), Yh, n_used=n_used, status=status)
+        ap.approxifer_decode(p, dirty.to(dev()), ap.mask_tensor(mask), Yh, n_used=n_used, status=status,
+                             tuning=ap.decode_tuning(kernel=2))
         if flags == 0:  # (the literal sign has poles: on arbitrary masks a denominator can vanish, see pin P9)
             check_decode(K, W, Yt, mask, Yh, n_used, status, flags)
         assert bool((guard[:32] == CANARY).all()) and bool((guard[32 + G * K * C:] == CANARY).all())
         ref = ap.approxifer_decode(p, dirty.to(dev()), ap.mask_tensor(mask), tuning=ap.decode_tuning(kernel=1))
         assert torch.equal(Yh.contiguous().view(torch.int32), ref.view(torch.int32))  # bit patterns: inf/NaN included
+
+
+PACK_SHAPES = [
+    # K, W, C, G
+    (8, 12, 10, 1000),    # the paper's shape: whole-block copies, 4 queries per thread, 5 words each
+    (8, 12, 10, 65),      # one full item and one group
+    (4, 5, 10, 7),        # a last item that ends on an 8-byte boundary
+    (5, 9, 10, 131),      # odd K: tiles of 2 queries
+    (3, 7, 20, 50),       # coincident nodes (rows copied), whole-block copies
+    (3, 7, 62, 50),       # coincident nodes, the longest rows this kernel takes
+    (1, 2, 2, 300),       # the smallest of everything: one word per row
+    (2, 5, 6, 257),
+    (7, 13, 46, 77),      # 23 words per row: a ragged split (3 threads x 8 words)
+    (12, 20, 36, 100),
+    (16, 24, 48, 300),
+    (8, 12, 64, 500),     # longer rows: other kernels (the comparison still holds)
+    (16, 24, 128, 70),
+    (32, 32, 20, 40),     # largest K and W: 16 lanes per group
+    (32, 32, 40, 9),      # 32 lanes per group: one group per item
+    (9, 24, 30, 64),
+    (12, 20, 10, 999),    # six lanes per group: five groups do not start on 16-byte boundaries, four do
+    (8, 24, 10, 333),
+    (16, 24, 10, 1000),
+]
+
+
+@pytest.mark.parametrize("K,W,C,G", PACK_SHAPES)
+def test_packed_groups_decoder_against_oracle_and_register_decoder(K, W, C, G):
+    """Dense buffers with an even number of classes up to 62 take the kernel in which every warp runs its own
+    pipeline over items of several groups.  It adds the same terms in the same order as the per-column kernel:
+    equal to the last bit; absent rows (NaN here) never used; both sign rules; a two-slot ring with five warps
+    and a four-slot ring with one-group items forced as well."""
+    rng = np.random.default_rng(K * 1000 + C)
+    Yt = torch.randn((G, W, C), generator=torch.Generator().manual_seed(C + K))
+    mask = random_masks(W, G, rng, min_present=0)
+    mask[0] = 0
+    mask[G - 1] = 2**W - 1
+    if G > 4:
+        mask[1], mask[2], mask[3] = 1, 1 << (W - 1), (2**W - 1) & ~2
+    dirty = Yt.clone()
+    for gi in range(G):
+        for i in range(W):
+            if not (int(mask[gi]) >> i) & 1:
+                dirty[gi, i] = float("nan")
+    dY, dm = dirty.to(dev()), ap.mask_tensor(mask)
+    for flags in (0, binding.SIGN_WORKER_INDEX):
+        p = ap.make_params(K, W, 0, flags)
+        ref = ap.approxifer_decode(p, dY, dm, tuning=ap.decode_tuning(kernel=1))
+        for tuning in (None, ap.decode_tuning(4, 2, 5, 0, 0), ap.decode_tuning(4, 4, 0, 1, 0)):
+            n_used = torch.empty(G, dtype=torch.int32, device=dev())
+            status = torch.empty(G, dtype=torch.int32, device=dev())
+            guard = torch.full((G * K * C + 64,), CANARY, device=dev())
+            Yh = guard[32: 32 + G * K * C].view(G, K, C)
+            ap.approxifer_decode(p, dY, dm, Yh, n_used=n_used, status=status, tuning=tuning)
+            if flags == 0:  # (the literal sign has poles on arbitrary masks, see pin P9)
+                check_decode(K, W, Yt, mask, Yh, n_used, status, flags)
+            assert bool((guard[:32] == CANARY).all()) and bool((guard[32 + G * K * C:] == CANARY).all())
+            assert torch.equal(Yh.contiguous().view(torch.int32), ref.view(torch.int32))  # bit patterns: inf/NaN included
+    assert ap.device_wait_timeouts() == 0
+
+
+def test_packed_groups_decoder_at_full_occupancy():
+    """Enough groups for every CTA to go several times round its ring (configs[1] shape, 20,000 groups)."""
+    K, W, C, G = 8, 12, 10, 20000
+    rng = np.random.default_rng(5)
+    Yt = torch.randn((G, W, C), generator=torch.Generator().manual_seed(9))
+    mask = random_masks(W, G, rng, min_present=8)
+    n_used = torch.empty(G, dtype=torch.int32, device=dev())
+    status = torch.empty(G, dtype=torch.int32, device=dev())
+    p = ap.make_params(K, W)
+    Yh = ap.approxifer_decode(p, Yt.to(dev()), ap.mask_tensor(mask), n_used=n_used, status=status)
+    check_decode(K, W, Yt, mask, Yh, n_used, status)
+    ref = ap.approxifer_decode(p, Yt.to(dev()), ap.mask_tensor(mask), tuning=ap.decode_tuning(kernel=1))
+    assert torch.equal(Yh, ref)
+    assert ap.device_wait_timeouts() == 0
 
 
 def test_worker_major_layouts_for_decode_and_locate():
