@@ -48,10 +48,11 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic (ncu dram__bytes_read.sum + dram__bytes_write.sum) of encode_kernel<12, float4, 768> per group of
 # the headline workload, from a capture of a reduced launch (profiles/encode_kernel_K12_W20_D150528.md); traffic is
-# proportional to the number of groups (every row is touched once).  None until the counters have been taken
-# for the kernel as it stands.
-ENCODE_TRAFFIC_PER_GROUP = None
-ENCODE_TRAFFIC_SOURCE = None
+# proportional to the number of groups (every row is touched once).  Set to None when the kernel changes, until
+# the counters have been taken again.
+ENCODE_TRAFFIC_PER_GROUP = (1387302912 + 2254066944) / 192
+ENCODE_TRAFFIC_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of a 192-group launch (3.7 GB) of the unchanged kernel, "
+                         "per group x groups; the written part misses the ~58 MB of dirty lines still in L2 at kernel end")
 E2E_GROUPS = 256
 CPU_SAMPLE_GROUPS = 64
 
@@ -277,6 +278,24 @@ def workload4_predictions(ap, dev, w4g):
     return Yt
 
 
+def decode3_alone_entry(ap, dev, peak, seed_offset=0, launches=30):
+    """The decoder alone on the headline workload's predictions (K=12, W=20, C=1000, 4,096 groups; 0.43 GB), launches
+    back to back.  Taken before the timed steps: a second of encoder steps at the board's power cap lowers the SM
+    clock, and a launch this short (its ramp-up and drain are a tenth of it) slows down with the clock."""
+    w3 = wl.workload(3)
+    p3 = ap.make_params(w3.K, w3.W)
+    Yt = wl.gaussian_predictions(w3, dev)
+    m3 = wl.masks(w3, seed_offset=seed_offset)
+    mt = ap.mask_tensor(m3, dev)
+    Yh = torch.empty((w3.G, w3.K, w3.C), device=dev)
+    times = []
+    time_launches(lambda: ap.approxifer_decode(p3, Yt, mt, Yh), 3, launches, times)
+    e = kernel_entry("decode_staged_kernel", HEADLINE_NAME + " (decoder timed alone before the steps, launches back to back)",
+                     decode_bytes(w3, m3), times, peak, w3.G)
+    del Yt, Yh
+    return e
+
+
 def decode4_entry(ap, dev, peak, launches=40):
     """The decoder alone on the largest decode workload (K=16, W=24, C=1000, 262,144 groups, 16-24 present)."""
     free, _ = torch.cuda.mem_get_info()
@@ -340,6 +359,17 @@ def decode_grid(ap, dev, gigabytes=3.0, worker_major=False):
             out.append(synthetic_decode(ap, dev, K, W, C, G, worker_major))
             torch.cuda.empty_cache()
     return out
+
+
+def fma_peak(ap, dev):
+    """fp32 multiply-add issue rate from a register-only loop (the second roof of the weighted sums)."""
+    sink = torch.zeros(1, device=dev)
+    iters, blocks = 4096, 148 * 8
+    med, mn = time_launches(lambda: ap.debug_fma_peak(iters, blocks, sink), 2, 5)
+    flop = 2.0 * 64 * iters * 256 * blocks
+    return {"fp32_fma_TFLOP_per_s": flop / mn / 1e9, "ms_min": mn, "ms_median": med,
+            "nominal_TFLOP_per_s": 148 * 128 * 2 * 1.965e9 / 1e12,
+            "note": "register-only loop, 16 independent chains per thread, 8 CTAs of 256 threads per SM; nominal = 148 SMs x 128 lanes x 2 x 1.965 GHz"}
 
 
 def host_cost(ap, dev):
@@ -460,6 +490,26 @@ def other_workloads(ap, dev, peak):
     Xt1 = torch.empty((w1.G, w1.W, w1.D), device=dev)
     med, mn = time_launches(lambda: ap.approxifer_encode(p1, X1, Xt1), 3, 20)
     entry("configs[0] encode K=4 W=5 D=784 (launch-latency bound, L2-resident)", encode_bytes(w1), med, mn, w1.G)
+    # bfloat16 payloads (fp32 weights and sums): bytes counted at 2 per element
+    w2b = wl.workload(2)
+    Xb = wl.queries(w2b, dev).to(torch.bfloat16)
+    Xtb = torch.empty((w2b.G, w2b.W, w2b.D), device=dev, dtype=torch.bfloat16)
+    p2b = ap.make_params(w2b.K, w2b.W)
+    med, mn = time_launches(lambda: ap.approxifer_encode_bf16(p2b, Xb, Xtb), 3, 20)
+    entry("configs[1] encode with bfloat16 payloads K=8 W=12 D=3072", encode_bytes(w2b) // 2, med, mn, w2b.G)
+    del Xb, Xtb
+    torch.cuda.empty_cache()
+    w4b = wl.workload(4, G=65536)
+    Ytb = workload4_predictions(ap, dev, w4b).to(torch.bfloat16)
+    m4b = wl.masks(w4b)
+    mtb = ap.mask_tensor(m4b, dev)
+    Yhb = torch.empty((w4b.G, w4b.K, w4b.C), device=dev, dtype=torch.bfloat16)
+    p4b = ap.make_params(w4b.K, w4b.W)
+    med, mn = time_launches(lambda: ap.approxifer_decode_bf16(p4b, Ytb, mtb, Yhb), 3, 10)
+    entry("configs[3] decode with bfloat16 payloads K=16 W=24 C=1000, 65536 groups (per-column kernel)",
+          2 * w4b.C * (present_workers(m4b) + w4b.K * w4b.G) + 4 * w4b.G, med, mn, w4b.G)
+    del Ytb, Yhb
+    torch.cuda.empty_cache()
     # the largest K and W the library takes
     G32 = 8192
     g = torch.Generator(device=dev)
@@ -490,6 +540,8 @@ def run_case(ap, dev, args):
         e = synthetic_decode(ap, dev, K, W, C, G, args.worker_major, iters, tuning)
         e.update(case="decode", dec_config=args.dec_config, wait_timeouts=ap.device_wait_timeouts())
         return e
+    if args.case == "fmapeak":
+        return {"case": "fmapeak", **fma_peak(ap, dev)}
     if args.case == "hostcost":
         return {"case": "hostcost", "calls": host_cost(ap, dev)}
     cfg = int(args.case[-1])
@@ -596,7 +648,7 @@ def main():
     ap_.add_argument("--groups", type=int, default=None, help="override the number of groups (profiling only)")
     ap_.add_argument("--case", default=None,
                      choices=["decode2", "decode3", "decode4", "decode5", "locate5", "locateh5", "rational5", "pair5", "encode2", "encode3",
-                              "decode", "grid", "hostcost"],
+                              "decode", "grid", "hostcost", "fmapeak"],
                      help="time one kernel alone (tuning / profiling) and print a short JSON line; `decode` takes --shape, "
                           "`grid` runs the decoder over payload lengths 10..256 on 3 GB problems")
     ap_.add_argument("--shape", default="8,12,64,1048576", help="K,W,C,G for --case decode")
@@ -633,6 +685,10 @@ def main():
         cpu = time_oracle()
 
     peak, peak_src = measured_peak()
+    # the small decode of the headline workload alone, before the long run of steps pulls the SM clock down
+    # (0.43 GB in ~76 us: at that size the kernel's ramp-up and drain depend on the clock)
+    dec3_alone = decode3_alone_entry(ap, dev, peak, seed_offset=rank) if (rank == 0 and args.groups is None) else None
+    torch.cuda.empty_cache()
     w_full = wl.workload(HEADLINE_CFG)
     free, _ = torch.cuda.mem_get_info()
     G = args.groups or fit_groups(w_full, 4 * w_full.D * (w_full.K + w_full.W) + 4 * w_full.C * (w_full.K + w_full.W) + 4,
@@ -692,9 +748,10 @@ def main():
 
     kernels = [
         kernel_entry("encode_kernel", HEADLINE_NAME + " (inside the timed steps)", enc_b, enc_times, peak, w.G),
-        kernel_entry("decode_staged_kernel", HEADLINE_NAME + " (inside the timed steps)", dec_b, dec_times, peak, w.G),
+        kernel_entry("decode_staged_kernel", HEADLINE_NAME + " (inside the timed steps, right after the encoder)", dec_b, dec_times, peak, w.G),
     ]
     if rank == 0 and args.groups is None:
+        kernels.append(dec3_alone)
         kernels.append(decode4_entry(ap, dev, peak))
 
     # end to end through the host-buffer entry points, on every rank (max over ranks, like the device figure)
@@ -730,6 +787,7 @@ def main():
         line["others"] = other_workloads(ap, dev, peak)
         line["decode_grid_3GB"] = decode_grid(ap, dev)
         line["host_cost"] = host_cost(ap, dev)
+        line["fma_peak"] = fma_peak(ap, dev)
     line.update({
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -72,6 +72,8 @@ extern "C" {
 #define APPROXIFER_ST_FEW_WORKERS 2u            /* decode: fewer than K workers present; computed anyway */
 #define APPROXIFER_ST_LOCATE_UNDERDETERMINED 4u /* locate: fewer than 2(K+E) workers present; nothing located */
 #define APPROXIFER_ST_NONFINITE 8u              /* locate: some Q(beta_i) was not finite (ranked as +inf) */
+#define APPROXIFER_ST_TIMEOUT 16u               /* decode: a bounded wait on a staged copy gave up before this group was finished;
+                                                   its output is unspecified (never set in a correct run) */
 
 /*
  * One params struct serves a whole encode -> locate -> decode pipeline: every entry point reads the fields
@@ -124,6 +126,26 @@ int approxifer_decode(const approxifer_params* params, int64_t G, int64_t C,
                       const uint32_t* mask,
                       float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
                       int32_t* n_used, uint32_t* status, void* cuda_stream);
+
+/*
+ * The encoder and the decoder on bfloat16 payloads: the same formulas (Section 3, "ApproxIFER Encoding" and
+ * "ApproxIFER Decoding", step 2), with X / Xt and Yt / Yhat holding bfloat16 elements (uint16_t bit patterns:
+ * the upper half of an IEEE-754 binary32), which halves the bytes the two memory-bound kernels move.  The paper
+ * fixes no storage precision; here a stored bfloat16 IS the number it denotes (widened exactly), weights and
+ * sums are fp32 exactly as in the fp32 entry points, and each result is rounded once to the nearest bfloat16,
+ * ties to even.  Strides are in ELEMENTS (of 2 bytes).  8-byte aligned bases with D (or C) and all strides
+ * multiples of 4 take the 64-bit path, anything else an element-wise one.  Arguments, mask, n_used, status and
+ * return codes as in approxifer_encode / approxifer_decode.
+ */
+int approxifer_encode_bf16(const approxifer_params* params, int64_t G, int64_t D,
+                           const uint16_t* X, int64_t x_gstride, int64_t x_rstride,
+                           uint16_t* Xt, int64_t xt_gstride, int64_t xt_rstride,
+                           void* cuda_stream);
+int approxifer_decode_bf16(const approxifer_params* params, int64_t G, int64_t C,
+                           const uint16_t* Yt, int64_t yt_gstride, int64_t yt_rstride,
+                           const uint32_t* mask,
+                           uint16_t* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                           int32_t* n_used, uint32_t* status, void* cuda_stream);
 
 /*
  * Byzantine-worker locator (Algorithm 2; Algorithm 1 is its inner step; the
@@ -290,11 +312,24 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
  *   `ctas_per_sm` bounds the warps per CTA and `cols` (any positive value) the groups per work item.
  * APPROXIFER_E_PARAM for any other value.
  *
+ * Exercising the bounded waits.  The two decoders that stage predictions with asynchronous copies (bulk-copy
+ * staged and packed-groups) bound every wait on such a copy and give up instead of hanging.  In a correct run
+ * no wait ever runs out, so the give-up path can only be reached on purpose: `withhold_group_plus1` = g + 1
+ * makes the kernel stage the work item that holds group g as usual but never announce it to the threads that
+ * wait for it, and `wait_limit` (>= 65536, so that copies already started have landed long before) replaces
+ * the built-in limit by that many non-blocking probes.  The waiting threads then give up after a few
+ * milliseconds: the CTA (bulk-copy staged) or the warp (packed-groups) that owned the item stops, writes
+ * APPROXIFER_ST_TIMEOUT into status[] of every group it has not finished (outputs of those groups are
+ * unspecified), counts the event (approxifer_device_wait_timeouts) and the kernel ends normally; all other
+ * groups are decoded as usual, and the context stays usable.  Nothing faults, traps or spins without limit.
+ *
  * force_warp_kernel != 0 routes the locate through the warp-per-group kernel, which otherwise serves only
  * K+E > 15 (smaller K+E use the thread-per-class kernel).  Both follow Algorithm 2 and return the same sets.
  */
 typedef struct approxifer_decode_tuning {
   int32_t kernel, stages, ctas_per_sm, cols, split;
+  uint32_t wait_limit;          /* see below; 0 = the built-in limit */
+  int64_t withhold_group_plus1; /* see below; 0 = none */
 } approxifer_decode_tuning;
 int approxifer_debug_decode(const approxifer_params* params, int64_t G, int64_t C,
                             const float* Yt, int64_t yt_gstride, int64_t yt_rstride,
@@ -309,12 +344,24 @@ int approxifer_debug_locate(const approxifer_params* params, int64_t G, int64_t 
                             int force_warp_kernel, void* cuda_stream);
 
 /*
+ * Measuring hook (not on the hot path; the paper has no counterpart): `blocks` CTAs of 256 threads each run
+ * `iters` rounds of 64 dependent-chain-free fp32 multiply-adds per thread on registers only (16 independent
+ * chains), 2 * 64 * iters * 256 * blocks flop in all.  Timed by the caller, it gives the issue rate of the plain
+ * fp32 pipe -- the second roof, next to HBM bandwidth, of the skinny weighted sums of Section 3 (2 K W / (4 (K + W))
+ * flop per payload byte).  `sink` is a device float that is never written in practice.
+ */
+int approxifer_debug_fma_peak(int iters, int blocks, float* sink, void* cuda_stream);
+
+/*
  * Every wait on an asynchronous copy inside the kernels is bounded.  Returns how
  * many such waits have given up on the current device since the library was
- * loaded (0 in a correct run; the affected groups' outputs are then
- * unspecified), or -1 if the counter cannot be read.  Synchronises the device.
+ * loaded or the counter was last reset (0 in a correct run; the affected groups
+ * carry APPROXIFER_ST_TIMEOUT in status[] and their outputs are unspecified), or
+ * -1 if the counter cannot be read.  Synchronises the device.
+ * approxifer_reset_device_wait_timeouts sets the counter back to 0.
  */
 int64_t approxifer_device_wait_timeouts(void);
+int approxifer_reset_device_wait_timeouts(void);
 
 /* Human-readable text for a return code (static storage). */
 const char* approxifer_strerror(int code);

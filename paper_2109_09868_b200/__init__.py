@@ -9,6 +9,8 @@ from .binding import (  # noqa: F401
     ApproxiferError,
     approxifer_debug_weights,
     approxifer_decode,
+    approxifer_decode_bf16,
+    approxifer_encode_bf16,
     approxifer_decode_rational,
     approxifer_encode,
     approxifer_encode_host,
@@ -20,7 +22,9 @@ from .binding import (  # noqa: F401
     approxifer_params,
     approxifer_decode_tuning,
     decode_tuning,
+    debug_fma_peak,
     device_wait_timeouts,
+    reset_device_wait_timeouts,
     launch_count,
     library_path,
     load,

@@ -22,7 +22,7 @@ E_NULL, E_RANGE, E_PARAM, E_CUDA, E_WORKSPACE, E_TOO_LARGE = -1, -2, -3, -4, -5,
 STATIC_WORKSPACE_BYTES = 32 << 20
 SIGN_RANK, SIGN_WORKER_INDEX = 0, 1
 LOCATE_HOMOGENEOUS = 2
-ST_NO_WORKERS, ST_FEW_WORKERS, ST_LOCATE_UNDERDETERMINED, ST_NONFINITE = 1, 2, 4, 8
+ST_NO_WORKERS, ST_FEW_WORKERS, ST_LOCATE_UNDERDETERMINED, ST_NONFINITE, ST_TIMEOUT = 1, 2, 4, 8, 16
 
 EXPORTS = (
     "approxifer_encode",
@@ -36,11 +36,15 @@ EXPORTS = (
     "approxifer_launch_count",
     "approxifer_debug_decode",
     "approxifer_device_wait_timeouts",
+    "approxifer_reset_device_wait_timeouts",
     "approxifer_debug_locate",
     "approxifer_encode_host",
     "approxifer_decode_host",
     "approxifer_locate_host",
     "approxifer_encode_host_static",
+    "approxifer_debug_fma_peak",
+    "approxifer_encode_bf16",
+    "approxifer_decode_bf16",
 )
 
 
@@ -49,7 +53,8 @@ class approxifer_params(ctypes.Structure):
 
 
 class approxifer_decode_tuning(ctypes.Structure):
-    _fields_ = [("kernel", c_int32), ("stages", c_int32), ("ctas_per_sm", c_int32), ("cols", c_int32), ("split", c_int32)]
+    _fields_ = [("kernel", c_int32), ("stages", c_int32), ("ctas_per_sm", c_int32), ("cols", c_int32), ("split", c_int32),
+                ("wait_limit", c_uint32), ("withhold_group_plus1", c_int64)]
 
 
 class ApproxiferError(RuntimeError):
@@ -86,6 +91,10 @@ def load() -> ctypes.CDLL:
     lib.approxifer_decode.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_int64,
                                       c_int64, c_void_p, c_void_p, c_void_p]
     lib.approxifer_decode.restype = c_int
+    lib.approxifer_encode_bf16.argtypes = lib.approxifer_encode.argtypes
+    lib.approxifer_encode_bf16.restype = c_int
+    lib.approxifer_decode_bf16.argtypes = lib.approxifer_decode.argtypes
+    lib.approxifer_decode_bf16.restype = c_int
     lib.approxifer_locate.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]
     lib.approxifer_locate.restype = c_int
@@ -105,6 +114,9 @@ def load() -> ctypes.CDLL:
                                             c_int64, c_void_p, c_void_p, POINTER(approxifer_decode_tuning), c_void_p]
     lib.approxifer_debug_decode.restype = c_int
     lib.approxifer_device_wait_timeouts.restype = c_int64
+    lib.approxifer_reset_device_wait_timeouts.restype = c_int
+    lib.approxifer_debug_fma_peak.argtypes = [c_int, c_int, c_void_p, c_void_p]
+    lib.approxifer_debug_fma_peak.restype = c_int
     lib.approxifer_debug_locate.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
                                             c_void_p, c_int, c_void_p]
     lib.approxifer_debug_locate.restype = c_int
@@ -136,13 +148,29 @@ def launch_count() -> int:
     return int(load().approxifer_launch_count())
 
 
-def decode_tuning(kernel: int = 0, stages: int = 0, ctas_per_sm: int = 0, cols: int = 0, split: int = 0) -> approxifer_decode_tuning:
-    """Per-call kernel choice / launch plan for approxifer_decode(..., tuning=...) (tests and tuning only)."""
-    return approxifer_decode_tuning(int(kernel), int(stages), int(ctas_per_sm), int(cols), int(split))
+def decode_tuning(kernel: int = 0, stages: int = 0, ctas_per_sm: int = 0, cols: int = 0, split: int = 0,
+                  wait_limit: int = 0, withhold_group: int = -1) -> approxifer_decode_tuning:
+    """Per-call kernel choice / launch plan for approxifer_decode(..., tuning=...) (tests and tuning only).
+    wait_limit / withhold_group exercise the kernels' bounded waits (see approxifer_debug_decode)."""
+    return approxifer_decode_tuning(int(kernel), int(stages), int(ctas_per_sm), int(cols), int(split), int(wait_limit),
+                                    int(withhold_group) + 1)
+
+
+def debug_fma_peak(iters: int, blocks: int, sink: torch.Tensor, stream=None) -> None:
+    """Register-only fp32 multiply-add loop (2 * 64 * iters * 256 * blocks flop); time it with CUDA events."""
+    rc = load().approxifer_debug_fma_peak(int(iters), int(blocks), sink.data_ptr(), _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_debug_fma_peak")
 
 
 def device_wait_timeouts() -> int:
     return int(load().approxifer_device_wait_timeouts())
+
+
+def reset_device_wait_timeouts() -> None:
+    rc = load().approxifer_reset_device_wait_timeouts()
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_reset_device_wait_timeouts")
 
 
 def make_params(K: int, W: int, E: int = 0, flags: int = 0) -> approxifer_params:
@@ -155,11 +183,11 @@ def _stream_ptr(stream) -> int:
     return int(stream.cuda_stream)
 
 
-def _payload(t: torch.Tensor, rows: int, name: str):
+def _payload(t: torch.Tensor, rows: int, name: str, dtype=torch.float32):
     if not t.is_cuda:
         raise ValueError("%s must be a CUDA tensor (the library has no CPU path)" % name)
-    if t.dtype != torch.float32 or t.dim() != 3 or t.shape[1] != rows:
-        raise ValueError("%s must be float32 [G][%d][L]" % (name, rows))
+    if t.dtype != dtype or t.dim() != 3 or t.shape[1] != rows:
+        raise ValueError("%s must be %s [G][%d][L]" % (name, dtype, rows))
     if t.shape[2] > 1 and t.stride(2) != 1:
         raise ValueError("%s: innermost dimension must be contiguous" % name)
     return t.data_ptr(), t.stride(0), t.stride(1)
@@ -186,6 +214,39 @@ def approxifer_encode(params: approxifer_params, X: torch.Tensor, Xt: Optional[t
     if rc != OK:
         raise ApproxiferError(rc, "approxifer_encode")
     return Xt
+
+
+def approxifer_encode_bf16(params: approxifer_params, X: torch.Tensor, Xt: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """bfloat16 X [G][K][D] -> bfloat16 coded queries Xt [G][W][D] (fp32 weights and sums, one rounding)."""
+    G, K, D = X.shape
+    if Xt is None:
+        Xt = torch.empty((G, params.W, D), device=X.device, dtype=torch.bfloat16)
+    xp, xg, xr = _payload(X, params.K, "X", torch.bfloat16)
+    op, og, orr = _payload(Xt, params.W, "Xt", torch.bfloat16)
+    if Xt.shape[0] != G or Xt.shape[2] != D:
+        raise ValueError("Xt must be [G][W][D]")
+    rc = load().approxifer_encode_bf16(ctypes.byref(params), G, D, xp, xg, xr, op, og, orr, _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_encode_bf16")
+    return Xt
+
+
+def approxifer_decode_bf16(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, Yhat: Optional[torch.Tensor] = None,
+                           n_used: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """bfloat16 Yt [G][W][C], mask [G] -> bfloat16 Yhat [G][K][C]."""
+    G, W, C = Yt.shape
+    if Yhat is None:
+        Yhat = torch.empty((G, params.K, C), device=Yt.device, dtype=torch.bfloat16)
+    yp, yg, yr = _payload(Yt, params.W, "Yt", torch.bfloat16)
+    op, og, orr = _payload(Yhat, params.K, "Yhat", torch.bfloat16)
+    if Yhat.shape[0] != G or Yhat.shape[2] != C:
+        raise ValueError("Yhat must be [G][K][C]")
+    rc = load().approxifer_decode_bf16(ctypes.byref(params), G, C, yp, yg, yr, _vec(mask, torch.int32, G, "mask"), op, og, orr,
+                                       _vec(n_used, torch.int32, G, "n_used"), _vec(status, torch.int32, G, "status"),
+                                       _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_decode_bf16")
+    return Yhat
 
 
 def approxifer_decode(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, Yhat: Optional[torch.Tensor] = None,

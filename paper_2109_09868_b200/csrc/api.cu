@@ -113,6 +113,35 @@ int approxifer_decode(const approxifer_params* params, int64_t G, int64_t C, con
                         DecodeTuning{}, cuda_stream);
 }
 
+int approxifer_encode_bf16(const approxifer_params* params, int64_t G, int64_t D, const uint16_t* X, int64_t x_gstride,
+                           int64_t x_rstride, uint16_t* Xt, int64_t xt_gstride, int64_t xt_rstride, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if ((rc = check_layout(G, D, x_rstride))) return rc;
+  if ((rc = check_layout(G, D, xt_rstride))) return rc;
+  if (x_gstride < 0 || xt_gstride < 0) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (X == nullptr || Xt == nullptr) return APPROXIFER_E_NULL;
+  EncodeArgs a{reinterpret_cast<const float*>(X), reinterpret_cast<float*>(Xt), x_gstride, x_rstride, xt_gstride, xt_rstride,
+               G, D, params->K, params->W, 1};
+  return from_cuda(launch_encode(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int approxifer_decode_bf16(const approxifer_params* params, int64_t G, int64_t C, const uint16_t* Yt, int64_t yt_gstride,
+                           int64_t yt_rstride, const uint32_t* mask, uint16_t* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                           int32_t* n_used, uint32_t* status, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if ((rc = check_layout(G, C, yt_rstride))) return rc;
+  if ((rc = check_layout(G, C, yh_rstride))) return rc;
+  if (yt_gstride < 0 || yh_gstride < 0) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (Yt == nullptr || Yhat == nullptr || mask == nullptr) return APPROXIFER_E_NULL;
+  DecodeArgs a{reinterpret_cast<const float*>(Yt), mask, reinterpret_cast<float*>(Yhat), n_used, status, yt_gstride, yt_rstride,
+               yh_gstride, yh_rstride, G, C, params->K, params->W, params->flags, DecodeTuning{}, 1};
+  return from_cuda(launch_decode(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
 int approxifer_debug_decode(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
                             int64_t yt_rstride, const uint32_t* mask, float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
                             int32_t* n_used, uint32_t* status, const approxifer_decode_tuning* tuning, void* cuda_stream) {
@@ -123,7 +152,11 @@ int approxifer_debug_decode(const approxifer_params* params, int64_t G, int64_t 
         cols < 0 || (tuning->kernel != 4 && cols != 0 && cols != 16 && cols != 32 && cols != 64 && cols != 128 && cols != 256) ||
         (split != 0 && split != 1 && split != 2 && split != 4))
       return APPROXIFER_E_PARAM;
+    if (tuning->wait_limit != 0 && tuning->wait_limit < 65536u) return APPROXIFER_E_PARAM;  // started copies need time to land
+    if (tuning->withhold_group_plus1 < 0) return APPROXIFER_E_PARAM;
     t.kernel = tuning->kernel, t.stages = tuning->stages, t.ctas_per_sm = tuning->ctas_per_sm, t.cols = cols, t.split = split;
+    t.wait_limit = tuning->wait_limit;
+    t.withhold_group = tuning->withhold_group_plus1 - 1;
   }
   return decode_checked(params, G, C, Yt, yt_gstride, yt_rstride, mask, Yhat, yh_gstride, yh_rstride, n_used, status, t,
                         cuda_stream);
@@ -184,6 +217,16 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
   if (w == nullptr || (which == 1 && (idx == nullptr || n == nullptr))) return APPROXIFER_E_NULL;
   return from_cuda(launch_debug_weights(params->K, params->W, params->flags, mask, which, w, idx, n,
                                         static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int approxifer_debug_fma_peak(int iters, int blocks, float* sink, void* cuda_stream) {
+  if (iters < 1 || blocks < 1 || blocks > (1 << 20)) return APPROXIFER_E_RANGE;
+  if (sink == nullptr) return APPROXIFER_E_NULL;
+  return from_cuda(launch_fma_peak(iters, blocks, sink, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int approxifer_reset_device_wait_timeouts(void) {
+  return (reset_decode_wait_timeouts() == cudaSuccess && reset_pack_wait_timeouts() == cudaSuccess) ? APPROXIFER_OK : APPROXIFER_E_CUDA;
 }
 
 int64_t approxifer_device_wait_timeouts(void) {

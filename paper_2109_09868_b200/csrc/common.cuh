@@ -14,16 +14,18 @@ constexpr uint32_t kStNoWorkers = 1u;
 constexpr uint32_t kStFewWorkers = 2u;
 constexpr uint32_t kStLocateUnderdetermined = 4u;
 constexpr uint32_t kStNonfinite = 8u;
+constexpr uint32_t kStTimeout = 16u;
 
 constexpr uint32_t kFlagSignWorkerIndex = 1u;
 constexpr uint32_t kFlagLocateHomogeneous = 2u;
 
 struct EncodeArgs {
-  const float* X;
+  const float* X;  // (bfloat16 payloads: really const uint16_t*, see `bf16`)
   float* Xt;
   int64_t x_gs, x_rs, o_gs, o_rs;  // element strides
   int64_t G, D;
   int32_t K, W;
+  int32_t bf16 = 0;  // payload elements are bfloat16 (2 bytes) instead of fp32; weights and sums stay fp32
 };
 
 // Test / tuning choices of one decode call (all zero = automatic); see approxifer_debug_decode.
@@ -34,6 +36,10 @@ struct DecodeTuning {
   int32_t ctas_per_sm = 0;  // ... upper bound on resident CTAs per SM
   int32_t cols = 0;         // ... 16-byte columns per work item
   int32_t split = 0;        // ... thread groups sharing the K queries of a column
+  // exercising the bounded waits (tests only): a poll limit (0 = the built-in one; polls are then non-blocking
+  // probes) and a group whose staged data is never announced to the threads that wait for it (-1 = none)
+  uint32_t wait_limit = 0;
+  int64_t withhold_group = -1;
 };
 
 struct DecodeArgs {
@@ -47,6 +53,7 @@ struct DecodeArgs {
   int32_t K, W;
   uint32_t flags;
   DecodeTuning tune = {};
+  int32_t bf16 = 0;  // Yt and Yh hold bfloat16 elements (2 bytes); weights and sums stay fp32
 };
 
 struct LocateArgs {
@@ -69,6 +76,7 @@ struct LocateArgs {
 cudaError_t launch_encode(const EncodeArgs& a, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
 cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream);
+cudaError_t launch_fma_peak(int iters, int blocks, float* sink, cudaStream_t stream);
 cudaError_t launch_debug_weights(int K, int W, uint32_t flags, uint32_t mask, int which, float* w, int32_t* idx,
                                  int32_t* n, cudaStream_t stream);
 
@@ -81,6 +89,8 @@ cudaError_t read_decode_wait_timeouts(unsigned int* out);
 bool decode_pack_eligible(const DecodeArgs& a);
 cudaError_t launch_decode_pack(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream);
 cudaError_t read_pack_wait_timeouts(unsigned int* out);
+cudaError_t reset_decode_wait_timeouts();
+cudaError_t reset_pack_wait_timeouts();
 
 // Short-payload decoder (C <= 32, dense buffers); see decode_small.cu.
 bool decode_small_eligible(const DecodeArgs& a);
@@ -116,6 +126,7 @@ cudaError_t ensure_dynamic_smem(Kernel kernel, int dev, int bytes) {
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7u) == 0; }
 
 #ifdef __CUDACC__
 // Streaming (evict-first) 128-bit and 32-bit global accesses: every payload
@@ -124,6 +135,48 @@ __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p);
 __device__ __forceinline__ float ld_stream(const float* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
 __device__ __forceinline__ void st_stream(float* p, float v) { __stcs(p, v); }
+
+// How a payload is stored and how a thread sees it: Store = what one access moves, Vec = its fp32 lanes.
+//   PayloadF32x4 / PayloadF32: fp32 elements, 16-byte / 4-byte columns
+//   PayloadBf16x4 / PayloadBf16: bfloat16 elements (the upper half of a binary32), 8-byte / 2-byte columns;
+//   widening is exact, narrowing rounds to nearest, ties to even (cvt.rn)
+struct PayloadF32x4 {
+  using Store = float4;
+  using Vec = float4;
+  static constexpr int kLanes = 4, kElemBytes = 4;
+  static __device__ __forceinline__ Vec load(const Store* p) { return __ldcs(p); }
+  static __device__ __forceinline__ void store(Store* p, Vec v) { __stcs(p, v); }
+};
+struct PayloadF32 {
+  using Store = float;
+  using Vec = float;
+  static constexpr int kLanes = 1, kElemBytes = 4;
+  static __device__ __forceinline__ Vec load(const Store* p) { return __ldcs(p); }
+  static __device__ __forceinline__ void store(Store* p, Vec v) { __stcs(p, v); }
+};
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+struct PayloadBf16x4 {
+  using Store = uint2;
+  using Vec = float4;
+  static constexpr int kLanes = 4, kElemBytes = 2;
+  static __device__ __forceinline__ Vec load(const Store* p) {
+    const uint2 u = __ldcs(p);
+    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                       __uint_as_float(u.y & 0xffff0000u));
+  }
+  static __device__ __forceinline__ void store(Store* p, Vec v) { __stcs(p, make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w))); }
+};
+struct PayloadBf16 {
+  using Store = unsigned short;
+  using Vec = float;
+  static constexpr int kLanes = 1, kElemBytes = 2;
+  static __device__ __forceinline__ Vec load(const Store* p) { return __uint_as_float((uint32_t)__ldcs(p) << 16); }
+  static __device__ __forceinline__ void store(Store* p, Vec v) { __stcs(p, (unsigned short)(pack_bf16x2(v, 0.f) & 0xffffu)); }
+};
 
 __device__ __forceinline__ uint32_t worker_bits(int W) { return W >= 32 ? 0xffffffffu : ((1u << W) - 1u); }
 #endif

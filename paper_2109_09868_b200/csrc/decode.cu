@@ -37,9 +37,11 @@ struct Vec<float> {
 // Generic decoder: one thread per (group, V-wide column).  Works for every
 // shape, alignment and mask; threads of one warp may belong to different
 // groups when C is small.
-template <int K, typename V>
+template <int K, typename P>
 __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_constant__ DecodeArgs a,
                                                                 const __grid_constant__ DecodeTables tab) {
+  using V = typename P::Vec;
+  using S = typename P::Store;
   using Ops = Vec<V>;
   constexpr int KP = (K + 3) / 4 * 4;              // table rows padded to whole float4s
   __shared__ __align__(16) float s_rg[kMaxW * KP];  // [i][j] = 1/(alpha_j - beta_i), 0 beyond K
@@ -60,7 +62,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
 
   const uint32_t mask = a.mask[g] & worker_bits(a.W);
   const int n = __popc(mask);
-  const V* in = reinterpret_cast<const V*>(a.Yt + g * a.y_gs) + v;
+  const S* in = reinterpret_cast<const S*>(reinterpret_cast<const unsigned char*>(a.Yt) + g * a.y_gs * P::kElemBytes) + v;
   const int64_t in_rs = a.y_rs / Ops::kLanes;
   const bool literal = (a.flags & kFlagSignWorkerIndex) != 0;
   const bool any_coin = tab.any_coin != 0;
@@ -114,7 +116,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
       V y[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u)
-        if ((bits >> u) & 1u) y[u] = ld_stream(in + (i0 + u) * in_rs);
+        if ((bits >> u) & 1u) y[u] = P::load(in + (i0 + u) * in_rs);
 #pragma unroll
       for (int u = 0; u < 8; ++u)
         if ((bits >> u) & 1u) {
@@ -136,7 +138,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u)
-        if (i[u] >= 0) y[u] = ld_stream(in + i[u] * in_rs);
+        if (i[u] >= 0) y[u] = P::load(in + i[u] * in_rs);
 #pragma unroll
       for (int u = 0; u < 4; ++u)
         if (i[u] >= 0) use_row(i[u], r + u, y[u]);
@@ -144,7 +146,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
     }
   }
 
-  V* out = reinterpret_cast<V*>(a.Yh + g * a.o_gs) + v;
+  S* out = reinterpret_cast<S*>(reinterpret_cast<unsigned char*>(a.Yh) + g * a.o_gs * P::kElemBytes) + v;
   const int64_t out_rs = a.o_rs / Ops::kLanes;
 #pragma unroll
   for (int j = 0; j < K; ++j) {
@@ -155,7 +157,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
       o = acc[j];
     else
       o = Ops::scale(__frcp_rn(den[j]), acc[j]);  // correctly rounded, like 1.0f / den
-    st_stream(out + j * out_rs, o);
+    P::store(out + j * out_rs, o);
   }
   if (v == 0) {
     if (a.n_used) a.n_used[g] = n;
@@ -165,7 +167,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
 
 template <int K, typename V>
 cudaError_t launch_one(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream) {
-  const int64_t Cv = a.C / Vec<V>::kLanes;
+  const int64_t Cv = a.C / V::kLanes;
   const int64_t items = a.G * Cv;
   const int64_t blocks = (items + kDecodeThreads - 1) / kDecodeThreads;
   if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
@@ -226,13 +228,16 @@ __global__ void debug_encode_weights_kernel(int K, int W, const __grid_constant_
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   const DecodeTables& tab = decode_tables(a.K, a.W);
-  const bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&
-                   a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  const bool by4 = a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 && a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  if (a.bf16) {  // bfloat16 payloads: the per-column kernel, four elements (8 bytes) per thread where it can
+    if (by4 && aligned8(a.Yt) && aligned8(a.Yh)) return dispatch_k<PayloadBf16x4>(a, tab, stream);
+    return dispatch_k<PayloadBf16>(a, tab, stream);
+  }
   if (decode_pack_eligible(a)) return launch_decode_pack(a, tab, stream);
   if (decode_small_eligible(a)) return launch_decode_small(a, tab, stream);
   if (decode_staged_eligible(a)) return launch_decode_staged(a, tab, stream);
-  if (vec) return dispatch_k<float4>(a, tab, stream);
-  return dispatch_k<float>(a, tab, stream);
+  if (by4 && aligned16(a.Yt) && aligned16(a.Yh)) return dispatch_k<PayloadF32x4>(a, tab, stream);
+  return dispatch_k<PayloadF32>(a, tab, stream);
 }
 
 cudaError_t launch_debug_weights(int K, int W, uint32_t flags, uint32_t mask, int which, float* w, int32_t* idx,

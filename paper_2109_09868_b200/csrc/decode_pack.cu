@@ -33,11 +33,10 @@ __device__ unsigned int g_pack_wait_timeouts = 0;  // bounded waits that gave up
 
 namespace {
 
-constexpr int kPackMaxWarps = 24;
-// warps per CTA by words per lane: short rows leave room for 24 warps of 80 registers, longer ones get 16 of 128
-__host__ __device__ constexpr int pack_max_warps(int nw) { return nw <= 5 ? kPackMaxWarps : 16; }
+constexpr int kPackMaxWarps = 24;  // 768 threads: 80 registers each
+__host__ __device__ constexpr int pack_max_warps(int) { return kPackMaxWarps; }
 constexpr int kPackMaxStages = 4;
-constexpr int kPackMaxNW = 10;  // words (float2) per thread and row
+constexpr int kPackMaxNW = 5;  // words (float2) per thread and row
 constexpr int kPackMaxC = 62;
 constexpr uint32_t kPackWaitLimit = 1u << 22;
 constexpr unsigned kFullMask = 0xffffffffu;
@@ -59,6 +58,19 @@ __device__ __forceinline__ bool p_try_wait(uint32_t bar, uint32_t parity) {
       "{\n"
       ".reg .pred p;\n"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool p_test_wait(uint32_t bar, uint32_t parity) {  // non-blocking probe
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
       "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(ok)
@@ -158,6 +170,8 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     const unsigned char* src = reinterpret_cast<const unsigned char*>(a.Yt + g0 * (int64_t)(W * C));
     unsigned char* dst = slots + (size_t)slot * plan.in_bytes;
     const uint32_t bar = p_smem_u32(full + slot);
+    // (test hook: the item that holds one chosen group is never fetched, so the wait for it runs out)
+    if (a.tune.withhold_group >= g0 && a.tune.withhold_group < g0 + ng) return;
     if (bytes16 != bytes) *reinterpret_cast<float2*>(dst + bytes16) = *reinterpret_cast<const float2*>(src + bytes16);
     p_arrive_expect_tx(bar, bytes16);  // (release: the two floats above are visible to whoever sees the phase complete)
     if (bytes16) p_bulk_g2s(p_smem_u32(dst), src, bytes16, bar);
@@ -168,6 +182,8 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     return (s < GW && g < a.G) ? (a.mask[g] & wb) : 0u;
   };
 
+  const bool probe = a.tune.wait_limit != 0;  // (test hook: a short limit, counted in non-blocking probes)
+  const uint32_t wait_limit = probe ? a.tune.wait_limit : kPackWaitLimit;
   // prologue: S-1 items in flight, their masks in registers (mq0 belongs to the item about to be reduced)
   const int64_t g_first = first * GW, g_stride = stride * GW;
   const int64_t g_end = g_first + my_items * g_stride;  // first group of the item after this warp's last
@@ -196,10 +212,14 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     {
       const uint32_t addr = p_smem_u32(full + slot);
       bool ok = false;
-      for (uint32_t it = 0; it < kPackWaitLimit && !ok; ++it) ok = p_try_wait(addr, parity);
+      for (uint32_t it = 0; it < wait_limit && !ok; ++it) ok = probe ? p_test_wait(addr, parity) : p_try_wait(addr, parity);
       if (!__all_sync(kFullMask, ok)) {
         if (lane == 0) atomicAdd(&g_pack_wait_timeouts, 1u);
         failed_g0 = g0;
+        // this warp's items from here on are not written: say so in their groups' status words
+        if (a.status != nullptr)
+          for (int64_t q = g0; q < g_end; q += g_stride)
+            if (s < GW && q + s < a.G) a.status[q + s] = kStTimeout;
         break;
       }
     }
@@ -216,7 +236,7 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
       uint32_t r = 0;  // present workers so far = rank of the next one
       const unsigned char* yr = yg;
       const unsigned char* wr = wrow0;
-#pragma unroll(NW <= 7 ? 2 : 1)
+#pragma unroll 2
       for (int i = 0; i < W; ++i, yr += row_bytes, wr += KP * 8) {
         uint64_t y[NW];
 #pragma unroll
@@ -299,8 +319,8 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     // shared memory is given up (bounded)
     for (int d = 0; d < S && failed_g0 + d * g_stride < g_end; ++d) {
       const uint32_t addr = p_smem_u32(full + slot);
-      for (uint32_t it = 0; it < kPackWaitLimit; ++it)
-        if (p_try_wait(addr, parity)) break;
+      for (uint32_t it = 0; it < wait_limit; ++it)
+        if (probe ? p_test_wait(addr, parity) : p_try_wait(addr, parity)) break;
       if (++slot == S) {
         slot = 0;
         parity ^= 1u;
@@ -314,14 +334,19 @@ struct PackChoice {
   int in_bytes = 0, table_bytes = 0, smem = 0;
 };
 
-// How the words of a row are dealt to lanes: NW words per lane, nch lanes per (group, query tile).  Exact splits
-// are preferred (no predicated tail), then more words per lane.
+// How the words of a row are dealt to lanes: NW <= 5 words per lane (more would need more registers than 24 warps
+// per SM leave), nch lanes per (group, query tile).  The largest NW that pads the row by at most an eighth, else the
+// one that pads it least.
 void choose_words(int Cw, int* nw, int* nch) {
   int best_nw = 1, best_waste = 1 << 30;
   for (int w = kPackMaxNW; w >= 1; --w) {
     const int n = (Cw + w - 1) / w;
     const int waste = n * w - Cw;
-    if (waste < best_waste && (w >= 4 || Cw < 4 || waste == 0)) best_nw = w, best_waste = waste;
+    if (waste * 8 <= Cw) {
+      best_nw = w;
+      break;
+    }
+    if (waste < best_waste) best_nw = w, best_waste = waste;
   }
   *nw = best_nw;
   *nch = (Cw + best_nw - 1) / best_nw;
@@ -398,15 +423,25 @@ cudaError_t dispatch_nw(const DecodeArgs& a, const DecodeTables& tab, const Pack
 
 }  // namespace
 
-// Dense buffers (rows and groups back to back), 16-byte aligned, an even number of classes up to 62.
+// Dense buffers (rows and groups back to back), 16-byte aligned, an even number of classes up to 62.  Chosen
+// automatically where it is the fastest of the decoders (measured on 2 GB problems, K = 4 .. 16: 1.25-1.3x the
+// thread-per-(query, chunk) kernel at C = 10): rows of 6 .. 10 classes, which one lane covers whole, and
+// problems beyond the L2 cache (on cache-resident ones the two are equal and launch-bound).  Other even C up
+// to 62 run correctly when asked for (tuning kernel = 4) but lose to the other kernels.
 bool decode_pack_eligible(const DecodeArgs& a) {
   if (a.tune.kernel != 0 && a.tune.kernel != 4) return false;
+  if (a.tune.kernel == 0 && (a.C < 6 || a.C > 2 * kPackMaxNW || a.G * (int64_t)a.W * a.C * 4 < (int64_t(64) << 20))) return false;
   if (a.y_rs != a.C || a.y_gs != (int64_t)a.W * a.C || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
   if (!aligned16(a.Yt) || !aligned16(a.Yh)) return false;
   const DeviceInfo* di = nullptr;
   if (current_device_info(&di) != cudaSuccess) return false;
   PackChoice c;
   return plan_pack(a, di->smem_per_sm, &c);
+}
+
+cudaError_t reset_pack_wait_timeouts() {
+  const unsigned int zero = 0;
+  return cudaMemcpyToSymbol(g_pack_wait_timeouts, &zero, sizeof(unsigned int));
 }
 
 cudaError_t read_pack_wait_timeouts(unsigned int* out) {

@@ -61,10 +61,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kWaitLimit attempts.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kWaitLimit; ++it)
-    if (mbar_try_wait(bar, parity)) return true;
+// Non-blocking probe of a phase (the test hook's short waits poll with this one, so that their length is a
+// number of probes and not a multiple of try_wait's system-dependent blocking time).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within `limit` attempts.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit, bool probe) {
+  for (uint32_t it = 0; it < limit; ++it)
+    if (probe ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return true;
   return false;
 }
 // 1-D bulk copy global -> this CTA's shared memory; src, dst and bytes are multiples of 16.
@@ -149,10 +164,12 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
   const int64_t my_items = first < plan.n_items ? (plan.n_items - first + stride - 1) / stride : 0;
 
   // Bounded wait that also gives up when another warp of the CTA has given up.
+  const bool probe = a.tune.wait_limit != 0;  // (test hook: a short limit, counted in non-blocking probes)
+  const uint32_t wait_limit = probe ? a.tune.wait_limit : kWaitLimit;
   auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
-      if (mbar_try_wait(addr, parity)) return true;
+    for (uint32_t it = 0; it < wait_limit; ++it) {
+      if (probe ? mbar_test_wait(addr, parity) : mbar_try_wait(addr, parity)) return true;
       if ((it & 255u) == 255u && *abort_flag) return false;
     }
     return false;
@@ -251,7 +268,8 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
         inv_den[lane] = 1.0f / d;
       }
       __syncwarp();  // the whole item block is written before lane 0 publishes it
-      if (lane == 0) mbar_arrive(bar);
+      // (test hook: the item of one chosen group is staged but never announced, so the waits for it run out)
+      if (lane == 0 && g != a.tune.withhold_group) mbar_arrive(bar);
       // next item of this CTA
       if (++stage == S) {
         stage = 0;
@@ -267,7 +285,8 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
     if (k < my_items) {
       // A wait gave up (here or in a compute warp).  Let the copies already started land (bounded), then leave.
       give_up();
-      for (int64_t q = (k > S ? k - S : 0); q < k; ++q) (void)mbar_wait(smem_u32(full + (q % S)), (uint32_t)((q / S) & 1));
+      for (int64_t q = (k > S ? k - S : 0); q < k; ++q)
+        (void)mbar_wait(smem_u32(full + (q % S)), (uint32_t)((q / S) & 1), wait_limit, probe);
     }
     return;
   }
@@ -280,6 +299,9 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
   for (int64_t k = 0; k < my_items; ++k) {
     if (!wait(full + stage, phase)) {
       give_up();
+      // this CTA's items from here on are not (fully) written: say so in their groups' status words
+      if (tid == 0 && a.status != nullptr)
+        for (int64_t q = k; q < my_items; ++q) a.status[(first + q * stride) / plan.tiles] = kStTimeout;
       return;
     }
     // the producer left the item's coordinates in the slot's header
@@ -492,6 +514,11 @@ cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, c
   if (taken) return e;
   if (a.tune.split == 4) return dispatch_kt<4>((a.K + 3) / 4, a, tab, stream);
   return dispatch_kt<2>((a.K + 1) / 2, a, tab, stream);
+}
+
+cudaError_t reset_decode_wait_timeouts() {
+  const unsigned int zero = 0;
+  return cudaMemcpyToSymbol(g_decode_wait_timeouts, &zero, sizeof(unsigned int));
 }
 
 cudaError_t read_decode_wait_timeouts(unsigned int* out) {

@@ -38,9 +38,11 @@ struct VecOps<float> {
 // One work item = (group g, column v) with v counting V-wide columns of the
 // payload; items are numbered g*Dv + v and dealt to threads in order, so a
 // warp reads and writes 32 consecutive columns of a row.
-template <int K, typename V, int THREADS>
+template <int K, typename P, int THREADS>
 __global__ void __launch_bounds__(THREADS) encode_kernel(const __grid_constant__ EncodeArgs a,
                                                          const __grid_constant__ EncodeTables tab) {
+  using V = typename P::Vec;
+  using S = typename P::Store;
   using Ops = VecOps<V>;
   const uint32_t Dv = (uint32_t)(a.D / Ops::kLanes);
   const int64_t first = (int64_t)blockIdx.x * THREADS;  // first item of this block
@@ -51,14 +53,14 @@ __global__ void __launch_bounds__(THREADS) encode_kernel(const __grid_constant__
   const int64_t g = g0 + dg;
   if (g >= a.G) return;
 
-  const V* in = reinterpret_cast<const V*>(a.X + g * a.x_gs) + v;
-  V* out = reinterpret_cast<V*>(a.Xt + g * a.o_gs) + v;
+  const S* in = reinterpret_cast<const S*>(reinterpret_cast<const unsigned char*>(a.X) + g * a.x_gs * P::kElemBytes) + v;
+  S* out = reinterpret_cast<S*>(reinterpret_cast<unsigned char*>(a.Xt) + g * a.o_gs * P::kElemBytes) + v;
   const int64_t in_rs = a.x_rs / Ops::kLanes;
   const int64_t out_rs = a.o_rs / Ops::kLanes;
 
   V x[K];
 #pragma unroll
-  for (int j = 0; j < K; ++j) x[j] = ld_stream(in + j * in_rs);
+  for (int j = 0; j < K; ++j) x[j] = P::load(in + j * in_rs);
 
   const int W = a.W;
   for (int i = 0; i < W; ++i) {
@@ -66,19 +68,20 @@ __global__ void __launch_bounds__(THREADS) encode_kernel(const __grid_constant__
     V acc = Ops::mul(wi[0], x[0]);
 #pragma unroll
     for (int j = 1; j < K; ++j) acc = Ops::fma(wi[j], x[j], acc);
-    st_stream(out + i * out_rs, acc);
+    P::store(out + i * out_rs, acc);
   }
 }
 
-template <int K, typename V>
+template <int K, typename P>
 cudaError_t launch_one(const EncodeArgs& a, const EncodeTables& tab, cudaStream_t stream) {
-  const int64_t Dv = a.D / VecOps<V>::kLanes;
+  using V = P;  // (the kernels are instantiated per payload policy)
+  const int64_t Dv = a.D / P::kLanes;
   const int64_t items = a.G * Dv;
   // Rows that tile exactly into pieces of 768 columns (12 KB: a whole row of a 3x32x32 query) get CTAs of that
   // size: each CTA then reads and writes whole contiguous pieces of K and W rows, which HBM serves slightly
   // better (+0.8 % on workload 2) than the 4 KB pieces of 256-thread CTAs.
   // (K <= 16: beyond that 768 threads do not leave a thread enough registers for its K inputs)
-  if constexpr (VecOps<V>::kLanes == 4 && K <= 16) {
+  if constexpr (P::kLanes == 4 && K <= 16) {
     if (Dv % kEncodeWideThreads == 0) {
       const int64_t blocks = items / kEncodeWideThreads;
       if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
@@ -104,15 +107,44 @@ cudaError_t dispatch_k(const EncodeArgs& a, const EncodeTables& tab, cudaStream_
   }
 }
 
+// Register-only fp32 multiply-add loop: 16 independent chains per thread, nothing but FFMA in the loop body.
+// Measures the issue rate of the plain fp32 pipe, the second roof of the skinny weighted sums (an encoder with
+// K = W = 32 needs 8 flop per payload byte).
+__global__ void __launch_bounds__(256) fma_peak_kernel(int iters, float seed, float* sink) {
+  float acc[16];
+#pragma unroll
+  for (int c = 0; c < 16; ++c) acc[c] = seed + (float)(threadIdx.x + c);
+  const float a = 1.0f + seed * 1e-7f, b = seed * 1e-9f;
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int rep = 0; rep < 4; ++rep)
+#pragma unroll
+      for (int c = 0; c < 16; ++c) acc[c] = fmaf(acc[c], a, b);
+  }
+  float total = 0.f;
+#pragma unroll
+  for (int c = 0; c < 16; ++c) total += acc[c];
+  if (total == 123.456f) *sink = total;  // (never true in practice; keeps the loop alive)
+}
+
 }  // namespace
+
+cudaError_t launch_fma_peak(int iters, int blocks, float* sink, cudaStream_t stream) {
+  fma_peak_kernel<<<blocks, 256, 0, stream>>>(iters, 1.0f, sink);
+  count_launch();
+  return cudaGetLastError();
+}
 
 cudaError_t launch_encode(const EncodeArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   const EncodeTables& tab = encode_tables(a.K, a.W);
-  const bool vec = aligned16(a.X) && aligned16(a.Xt) && a.D % 4 == 0 && a.x_gs % 4 == 0 && a.x_rs % 4 == 0 &&
-                   a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
-  if (vec) return dispatch_k<float4>(a, tab, stream);
-  return dispatch_k<float>(a, tab, stream);
+  const bool by4 = a.D % 4 == 0 && a.x_gs % 4 == 0 && a.x_rs % 4 == 0 && a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  if (a.bf16) {  // four bfloat16 elements are one 8-byte column
+    if (by4 && aligned8(a.X) && aligned8(a.Xt)) return dispatch_k<PayloadBf16x4>(a, tab, stream);
+    return dispatch_k<PayloadBf16>(a, tab, stream);
+  }
+  if (by4 && aligned16(a.X) && aligned16(a.Xt)) return dispatch_k<PayloadF32x4>(a, tab, stream);
+  return dispatch_k<PayloadF32>(a, tab, stream);
 }
 
 }  // namespace approxifer

@@ -22,7 +22,8 @@ import torch
 from . import binding as ap
 
 
-def run_cell(K: int, S: int, E: int, sigma: float, softmax: bool, G: int, C: int, d_in: int, seed: int, dev) -> dict:
+def run_cell(K: int, S: int, E: int, sigma: float, softmax: bool, G: int, C: int, d_in: int, seed: int, dev,
+             keep_tensors: bool = False) -> dict:
     W = 2 * (K + E) + S if E > 0 else K + S
     gen = torch.Generator(device=dev)
     gen.manual_seed(seed)
@@ -50,7 +51,7 @@ def run_cell(K: int, S: int, E: int, sigma: float, softmax: bool, G: int, C: int
         adv, trusted = ap.approxifer_locate(p, Yt, ap.mask_tensor(mask, dev))
         recall = float((adv.cpu().numpy() == bad).all(axis=1).mean())
     else:
-        trusted, recall = ap.mask_tensor(mask, dev), float("nan")
+        adv, trusted, recall = None, ap.mask_tensor(mask, dev), float("nan")
     Yh = ap.approxifer_decode(p, Yt, trusted)
     Y = f(X)
     err = (Yh - Y).abs().amax(dim=(1, 2)) / Y.abs().amax(dim=(1, 2))
@@ -58,6 +59,8 @@ def run_cell(K: int, S: int, E: int, sigma: float, softmax: bool, G: int, C: int
     out = {"K": K, "S": S, "E": E, "W": W, "sigma": sigma, "model": "softmax" if softmax else "linear",
            "located_equals_injected": recall, "decode_rel_err_median": float(err.median()),
            "decode_rel_err_max": float(err.max()), "argmax_agreement": agree}
+    if keep_tensors:  # (for the tests: what went into and came out of the library)
+        out["tensors"] = {"Yt": Yt, "mask": mask, "injected": bad, "adv": adv, "trusted": trusted, "Yhat": Yh}
     if 2 <= K + E <= 13 and 2 * (K + E) <= W:
         # Algorithm 3 on the same corrupted predictions: P/Q at the alpha nodes, nothing located
         Yr = ap.approxifer_decode_rational(p, Yt, ap.mask_tensor(mask, dev))

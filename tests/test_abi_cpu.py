@@ -18,7 +18,7 @@ HEADER = os.path.join(ROOT, "include", "approxifer.h")
 def _declared_symbols():
     text = open(HEADER).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(approxifer_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(approxifer_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():
@@ -105,10 +105,15 @@ def test_debug_entry_points_validate_their_tuning_on_the_host():
     for (fields, want) in [((0, 0, 0, 0, 0), binding.OK), ((1, 0, 0, 0, 0), binding.OK), ((5, 0, 0, 0, 0), binding.E_PARAM), ((4, 0, 0, 7, 0), binding.OK),
                            ((0, 1, 0, 0, 0), binding.E_PARAM), ((0, 0, -1, 0, 0), binding.E_PARAM), ((0, 0, 0, 48, 0), binding.E_PARAM),
                            ((0, 0, 0, 0, 3), binding.E_PARAM), ((0, 4, 2, 256, 2), binding.OK)]:
-        t = binding.approxifer_decode_tuning(*fields)
+        t = binding.approxifer_decode_tuning(*fields, 0, 0)
         rc = lib.approxifer_debug_decode(ctypes.byref(p), 0, 64, None, 768, 64, None, None, 512, 64, None, None, ctypes.byref(t), None)
         assert rc == want, fields
     assert lib.approxifer_debug_decode(ctypes.byref(p), 0, 64, None, 768, 64, None, None, 512, 64, None, None, None, None) == binding.OK
+    # a poll limit too short for started copies to land, or a negative group, is refused
+    for (limit, withhold, want) in [(65536, 5, binding.OK), (1000, 0, binding.E_PARAM), (0, -1, binding.E_PARAM)]:
+        t = binding.approxifer_decode_tuning(0, 0, 0, 0, 0, limit, withhold)
+        rc = lib.approxifer_debug_decode(ctypes.byref(p), 0, 64, None, 768, 64, None, None, 512, 64, None, None, ctypes.byref(t), None)
+        assert rc == want, (limit, withhold)
     q = ap.make_params(8, 24, 2)
     assert lib.approxifer_debug_locate(ctypes.byref(q), 0, 10, None, 240, 10, None, None, None, None, 1, None) == binding.OK
     q = ap.make_params(8, 19, 2)

@@ -519,8 +519,9 @@ def test_packed_groups_decoder_against_oracle_and_register_decoder(K, W, C, G):
 
 
 def test_packed_groups_decoder_at_full_occupancy():
-    """Enough groups for every CTA to go several times round its ring (configs[1] shape, 20,000 groups)."""
-    K, W, C, G = 8, 12, 10, 20000
+    """A problem beyond the L2 cache, where this kernel is the automatic choice and every warp goes several times
+    round its ring (configs[1] shape, 160,000 groups)."""
+    K, W, C, G = 8, 12, 10, 160000
     rng = np.random.default_rng(5)
     Yt = torch.randn((G, W, C), generator=torch.Generator().manual_seed(9))
     mask = random_masks(W, G, rng, min_present=8)
