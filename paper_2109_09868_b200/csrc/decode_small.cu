@@ -1,6 +1,6 @@
 // ApproxIFER decoder, short- and medium-payload variant (Section 3, "Decoding", step 2) for predictions of
 // up to a few hundred classes (the paper's own workloads have C = 10; 100 classes is the next common size) in
-// dense [G][W][C] / [G][K][C] buffers.
+// dense [G][W][C] / [G][K][C] buffers (the predictions may also be stored worker-major, [W][G][C]).
 //
 // Same arithmetic as decode_kernel, term by term and rounding by rounding, but one thread per
 // (group, QUERY, chunk of CP <= 32 classes) instead of one per (group, 16-byte column): the thread walks the
@@ -41,14 +41,37 @@ __global__ void __launch_bounds__(kSmallThreads) decode_small_kernel(const __gri
   float* rgs = os + ((gpb * K * C + 3) & ~3);
   uint32_t* masks = reinterpret_cast<uint32_t*>(rgs + W * K);
 
-  // ---- stage: predictions (dense, so one contiguous range), table, masks ------------------------------
+  // ---- stage: predictions, table, masks --------------------------------------------------------------
   {
-    const float4* src = reinterpret_cast<const float4*>(a.Yt + g_first * a.y_gs);
-    float4* dst = reinterpret_cast<float4*>(ys);
-    const int n4 = in_floats >> 2;  // every CTA's range starts on a 16-byte boundary: whole float4s ...
-    for (int idx = tid; idx < n4; idx += kSmallThreads) dst[idx] = ld_stream(src + idx);
-    for (int idx = (n4 << 2) + tid; idx < in_floats; idx += kSmallThreads)  // ... except at the end of the last CTA
-      ys[idx] = ld_stream(a.Yt + g_first * a.y_gs + idx);
+    if (a.y_rs == a.C) {
+      // group-major ([G][W][C] dense): the CTA's groups are one contiguous range
+      const float4* src = reinterpret_cast<const float4*>(a.Yt + g_first * a.y_gs);
+      float4* dst = reinterpret_cast<float4*>(ys);
+      const int n4 = in_floats >> 2;  // every CTA's range starts on a 16-byte boundary: whole float4s ...
+      for (int idx = tid; idx < n4; idx += kSmallThreads) dst[idx] = ld_stream(src + idx);
+      for (int idx = (n4 << 2) + tid; idx < in_floats; idx += kSmallThreads)  // ... except at the end of the last CTA
+        ys[idx] = ld_stream(a.Yt + g_first * a.y_gs + idx);
+    } else {
+      // worker-major ([W][G][C]: y_gs == C, one batch per worker): W contiguous ranges of ng * C floats, read
+      // with 128-bit loads where they are whole 16-byte columns and scattered into the group-major layout
+      const int per_worker = ng * C;
+      const int n4 = per_worker >> 2;
+      for (int idx = tid; idx < W * n4; idx += kSmallThreads) {
+        const int i = idx / n4, q = idx - i * n4;
+        const float4 v = ld_stream(reinterpret_cast<const float4*>(a.Yt + (int64_t)i * a.y_rs + g_first * (int64_t)C) + q);
+        const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const int f = 4 * q + t, sgrp = f / C, c = f - sgrp * C;
+          ys[(sgrp * W + i) * C + c] = e[t];
+        }
+      }
+      const int rem = per_worker - (n4 << 2);  // ragged end of the last CTA
+      for (int idx = tid; idx < W * rem; idx += kSmallThreads) {
+        const int i = idx / rem, f = (n4 << 2) + idx - i * rem, sgrp = f / C, c = f - sgrp * C;
+        ys[(sgrp * W + i) * C + c] = ld_stream(a.Yt + (int64_t)i * a.y_rs + g_first * (int64_t)C + f);
+      }
+    }
     for (int idx = tid; idx < W * K; idx += kSmallThreads) rgs[idx] = tab.rg[idx];
     if (tid < ng) masks[tid] = a.mask[g_first + tid] & worker_bits(W);
   }
@@ -175,7 +198,7 @@ int groups_per_cta(const DecodeArgs& a, const ChunkPlan& p) {
   while (gpb > 0 && gpb * per_group + fixed > kSmallSmemBudget) --gpb;
   // every CTA's ranges must start on 16-byte boundaries: any number of groups if a group is whole float4s,
   // else a multiple of 4 groups
-  if (((int64_t)a.W * C) % 4 != 0 || ((int64_t)a.K * C) % 4 != 0) gpb &= ~3;
+  if (((int64_t)a.W * C) % 4 != 0 || ((int64_t)a.K * C) % 4 != 0 || (a.y_rs != a.C && C % 4 != 0)) gpb &= ~3;
   return gpb;
 }
 
@@ -220,7 +243,11 @@ cudaError_t dispatch_cp(const DecodeArgs& a, const DecodeTables& tab, const Chun
 // plan_chunks), and room for at least one group per CTA.
 bool decode_small_eligible(const DecodeArgs& a) {
   if (a.tune.kernel != 0 && a.tune.kernel != 2) return false;
-  if (a.y_rs != a.C || a.y_gs != (int64_t)a.W * a.C || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
+  // predictions group-major and dense, or worker-major ([W][G][C]: groups C apart, workers' batches whole
+  // 16-byte columns apart); results dense
+  const bool group_major = a.y_rs == a.C && a.y_gs == (int64_t)a.W * a.C;
+  const bool worker_major = a.y_gs == a.C && a.y_rs >= a.G * a.C && a.y_rs % 4 == 0;
+  if (!(group_major || worker_major) || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
   if (!aligned16(a.Yt) || !aligned16(a.Yh)) return false;
   const ChunkPlan p = plan_chunks(a.C);
   if (p.cp == 0 || a.K * p.nch > kSmallThreads) return false;

@@ -552,6 +552,24 @@ def test_worker_major_layouts_for_decode_and_locate():
         check_decode(K, W, Yt, ref["trusted"], out.permute(1, 0, 2))
 
 
+@pytest.mark.parametrize("K,W,C,G", [(8, 12, 10, 1001), (8, 24, 10, 333), (16, 24, 31, 70), (3, 7, 9, 130), (12, 20, 36, 50), (4, 5, 2, 7)])
+def test_short_payload_decoder_reads_worker_major_predictions(K, W, C, G):
+    """Predictions stored one batch per worker ([W][G][C]) with dense results: the thread-per-(query, chunk) kernel
+    gathers the W ranges of a CTA's groups itself.  Bit-equal to the per-column kernel on the same view."""
+    rng = np.random.default_rng(K + C)
+    Yt = torch.randn((G, W, C), generator=torch.Generator().manual_seed(C))
+    mask = random_masks(W, G, rng, min_present=0)
+    wm = Yt.to(dev()).permute(1, 0, 2).contiguous()           # [W][G][C]
+    view = wm.permute(1, 0, 2)                                # [G][W][C] view: gstride = C, rstride = G*C
+    p = ap.make_params(K, W)
+    n_used = torch.empty(G, dtype=torch.int32, device=dev())
+    status = torch.empty(G, dtype=torch.int32, device=dev())
+    Yh = ap.approxifer_decode(p, view, ap.mask_tensor(mask), n_used=n_used, status=status)
+    check_decode(K, W, Yt, mask, Yh, n_used, status)
+    ref = ap.approxifer_decode(p, view, ap.mask_tensor(mask), tuning=ap.decode_tuning(kernel=1))
+    assert torch.equal(Yh.view(torch.int32), ref.view(torch.int32))
+
+
 @pytest.mark.parametrize("K,E,S,W,C", [(8, 2, 2, 24, 10), (3, 2, 1, 12, 37), (4, 1, 2, 12, 300), (2, 1, 0, 6, 1), (7, 3, 1, 22, 10),
                                        (10, 1, 0, 22, 10), (10, 2, 3, 27, 10), (12, 1, 0, 26, 10), (10, 3, 2, 28, 7), (11, 2, 6, 32, 10),
                                        (9, 2, 1, 23, 140), (12, 2, 0, 28, 10), (12, 3, 1, 31, 10), (13, 2, 2, 32, 5)])
