@@ -506,7 +506,7 @@ def other_workloads(ap, dev, peak):
     Yhb = torch.empty((w4b.G, w4b.K, w4b.C), device=dev, dtype=torch.bfloat16)
     p4b = ap.make_params(w4b.K, w4b.W)
     med, mn = time_launches(lambda: ap.approxifer_decode_bf16(p4b, Ytb, mtb, Yhb), 3, 10)
-    entry("configs[3] decode with bfloat16 payloads K=16 W=24 C=1000, 65536 groups (per-column kernel)",
+    entry("configs[3] decode with bfloat16 payloads K=16 W=24 C=1000, 65536 groups",
           2 * w4b.C * (present_workers(m4b) + w4b.K * w4b.G) + 4 * w4b.G, med, mn, w4b.G)
     del Ytb, Yhb
     torch.cuda.empty_cache()

@@ -229,7 +229,9 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   const DecodeTables& tab = decode_tables(a.K, a.W);
   const bool by4 = a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 && a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
-  if (a.bf16) {  // bfloat16 payloads: the per-column kernel, four elements (8 bytes) per thread where it can
+  if (a.bf16) {  // bfloat16 payloads: the bulk-copy staged kernel for long rows, else the per-column kernel, four
+                 // elements (8 bytes) per thread where it can
+    if (decode_staged_eligible(a)) return launch_decode_staged(a, tab, stream);
     if (by4 && aligned8(a.Yt) && aligned8(a.Yh)) return dispatch_k<PayloadBf16x4>(a, tab, stream);
     return dispatch_k<PayloadBf16>(a, tab, stream);
   }

@@ -22,6 +22,8 @@
 // through "full" / "empty" mbarriers, so producer and compute warps never meet
 // at a CTA-wide barrier.  Every wait is bounded.  Items are dealt round-robin
 // to the CTAs.  Every copy targets the issuing CTA's own shared memory.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace approxifer {
@@ -114,7 +116,8 @@ __host__ __device__ constexpr int ktp4(int KT) { return (KT + 3) / 4 * 4;  }  //
 __host__ __device__ constexpr int meta_bytes(int W, int KT, int SPLIT) { return (kWeightsOff + W * SPLIT * ktp4(KT) * 4 + 127) / 128 * 128; }
 constexpr int kTableOff = 128;  // float rg[W][K] after the mbarriers and the abort flag
 __host__ __device__ constexpr int slots_off(int W, int K) { return (kTableOff + W * (K | 1) * 4 + 127) / 128 * 128; }
-__host__ __device__ constexpr int slot_bytes(int W, int KT, int SPLIT, int COLS) { return meta_bytes(W, KT, SPLIT) + W * COLS * 16; }
+// (cb: bytes of a column of four elements -- 16 for fp32 payloads, 8 for bfloat16)
+__host__ __device__ constexpr int slot_bytes(int W, int KT, int SPLIT, int COLS, int cb = 16) { return meta_bytes(W, KT, SPLIT) + W * COLS * cb; }
 __host__ __device__ constexpr int min_ctas(int KT, int threads) {
   return KT > 8 ? 1 : (threads <= 64 ? 10 : (threads <= 96 ? 6 : (threads <= 160 ? 4 : (threads <= 288 ? 2 : 1))));
 }
@@ -122,15 +125,19 @@ __host__ __device__ constexpr int min_ctas(int KT, int threads) {
 // Shared memory: full[4] empty[4] mbarriers, abort flag | rg[W][K] | S slots, each = item block + W rows of COLS*16 B.
 // The producer compacts on the way in: the r-th PRESENT worker's row lands in row r of the slot and its signed
 // weights in row r of the item block, so the compute threads index both by rank with constant strides.
-template <int KT, int COLS, int SPLIT>
+// BF16: the payload elements are bfloat16 (a column of four is 8 bytes); they are widened exactly on their way
+// out of shared memory and the results rounded to nearest-even on their way out, everything between is the same.
+template <int KT, int COLS, int SPLIT, bool BF16 = false>
 __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 32))
     decode_staged_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ DecodeTables tab,
                          const __grid_constant__ StagedPlan plan) {
+  constexpr uint32_t CB = BF16 ? 8u : 16u;   // bytes of a column of four elements
+  constexpr int ES = BF16 ? 2 : 4;           // bytes of an element
   constexpr int KTP4 = ktp4(KT);
   constexpr int NP = KTP4 / 2;                   // query pairs per thread
   constexpr int kThreads = SPLIT * COLS;         // compute threads
   constexpr int kConsumerWarps = kThreads / 32;
-  constexpr uint32_t kRowBytes = COLS * 16u;     // one worker's row inside a ring slot
+  constexpr uint32_t kRowBytes = COLS * CB;      // one worker's row inside a ring slot
   constexpr int kWRowF = SPLIT * KTP4;           // floats of one rank's weights
   extern __shared__ __align__(128) unsigned char smem_raw[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
@@ -143,7 +150,7 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
   const uint32_t wb = worker_bits(W);
   const uint32_t Cv = (uint32_t)(a.C / 4);
   unsigned char* slots = smem_raw + slots_off(W, K);
-  const uint32_t slot_sz = (uint32_t)slot_bytes(W, KT, SPLIT, COLS);
+  const uint32_t slot_sz = (uint32_t)slot_bytes(W, KT, SPLIT, COLS, (int)CB);
   const uint32_t meta_sz = (uint32_t)meta_bytes(W, KT, SPLIT);
   const bool producer = warp == kConsumerWarps;  // the last warp moves data and prepares items; the others compute
   const bool literal = (a.flags & kFlagSignWorkerIndex) != 0;
@@ -210,7 +217,7 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
       }
       if (k >= S && !wait(empty + stage, phase)) break;  // compute warps are done with the slot
       const uint32_t col0 = (uint32_t)tile * COLS;
-      const uint32_t row_bytes = min((uint32_t)COLS, Cv - col0) * 16u;
+      const uint32_t row_bytes = min((uint32_t)COLS, Cv - col0) * CB;
       unsigned char* mb = slots + (size_t)stage * slot_sz;
       int32_t* hdr = reinterpret_cast<int32_t*>(mb);  // [0] = n, [1] = first column, [2..3] = group
       float* inv_den = reinterpret_cast<float*>(mb + 16);
@@ -224,7 +231,7 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
       if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)n * row_bytes);
       __syncwarp();
       if (present) {
-        const float* src = a.Yt + g * a.y_gs + (int64_t)lane * a.y_rs + (int64_t)col0 * 4;
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(a.Yt) + (g * a.y_gs + (int64_t)lane * a.y_rs + (int64_t)col0 * 4) * ES;
         bulk_g2s(smem_u32(mb) + meta_sz + (uint32_t)rank * kRowBytes, src, row_bytes, bar);
       }
       // 2. signed weights by rank, lane = worker: w[rank][c] = +-rg[i][j(c)].  The column is rotated by the
@@ -314,7 +321,12 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
     const float* inv_den = reinterpret_cast<const float*>(mb + 16);
     // idle threads (beyond the last column) shadow column 0 and store nothing
     const bool active = col < ncols;
-    const uint4* yp = reinterpret_cast<const uint4*>(mb + meta_sz) + (active ? col : 0u);               // + r * COLS
+    using Col = typename std::conditional<BF16, uint2, uint4>::type;  // a column of four payload elements as stored
+    auto widen = [](Col c) -> uint4 {  // ... and as the four fp32 bit patterns the arithmetic uses
+      if constexpr (BF16) return make_uint4(c.x << 16, c.x & 0xffff0000u, c.y << 16, c.y & 0xffff0000u);
+      else return c;
+    };
+    const Col* yp = reinterpret_cast<const Col*>(mb + meta_sz) + (active ? col : 0u);                    // + r * COLS
     const ulonglong2* wp = reinterpret_cast<const ulonglong2*>(mb + kWeightsOff) + half * (KTP4 / 4);  // + r * kWRowF / 4
 
     // acc[p][e] = (numerator of query 2p, numerator of query 2p+1) for payload element e of this column
@@ -326,13 +338,13 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
 
     if (n > 0) {
       // software pipeline over the ranks: the next row's payload and weights are loaded before this row's FMAs
-      uint4 yn = yp[0];
+      Col yn = yp[0];
       ulonglong2 wn[KTP4 / 4];
 #pragma unroll
       for (int q = 0; q < KTP4 / 4; ++q) wn[q] = wp[q];
 #pragma unroll 2
       for (int r = 0; r < n; ++r) {
-        const uint4 y = yn;
+        const uint4 y = widen(yn);
         uint64_t wpair[NP];
 #pragma unroll
         for (int q = 0; q < KTP4 / 4; ++q) {
@@ -365,7 +377,7 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
       phase ^= 1u;
     }
 
-    float4* out = reinterpret_cast<float4*>(a.Yh + g * a.o_gs) + col0 + col;
+    Col* out = reinterpret_cast<Col*>(reinterpret_cast<unsigned char*>(a.Yh) + g * a.o_gs * ES) + col0 + col;
     const int64_t out_rs = a.o_rs / 4;
 #pragma unroll
     for (int jj = 0; jj < KT; ++jj) {
@@ -378,19 +390,20 @@ __global__ void __launch_bounds__(SPLIT* COLS + 32, min_ctas(KT, SPLIT* COLS + 3
         else
           o = make_float4(inv[jj] * lo_f(acc[p][0]), inv[jj] * lo_f(acc[p][1]), inv[jj] * lo_f(acc[p][2]), inv[jj] * lo_f(acc[p][3]));
         if (n == 0) o = make_float4(0.f, 0.f, 0.f, 0.f);
-        st_stream(out + j * out_rs, o);
+        if constexpr (BF16) __stcs(out + j * out_rs, make_uint2(pack_bf16x2(o.x, o.y), pack_bf16x2(o.z, o.w)));
+        else st_stream(reinterpret_cast<float4*>(out + j * out_rs), o);
       }
     }
   }
 }
 
-template <int KT, int COLS, int SPLIT>
+template <int KT, int COLS, int SPLIT, bool BF16 = false>
 cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream) {
   const int64_t Cv = a.C / 4;
   StagedPlan plan;
   plan.tiles = (int32_t)((Cv + COLS - 1) / COLS);
   plan.n_items = a.G * plan.tiles;
-  const int64_t slot = slot_bytes(a.W, KT, SPLIT, COLS);
+  const int64_t slot = slot_bytes(a.W, KT, SPLIT, COLS, BF16 ? 8 : 16);
 
   const DeviceInfo* di = nullptr;
   cudaError_t e = current_device_info(&di);
@@ -412,8 +425,8 @@ cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t
   if (grid > plan.n_items) grid = plan.n_items;
 
   struct Tag {};
-  if ((e = ensure_dynamic_smem<Tag>(decode_staged_kernel<KT, COLS, SPLIT>, di->ordinal, (int)smem)) != cudaSuccess) return e;
-  decode_staged_kernel<KT, COLS, SPLIT><<<(unsigned)grid, SPLIT * COLS + 32, smem, stream>>>(a, tab, plan);
+  if ((e = ensure_dynamic_smem<Tag>(decode_staged_kernel<KT, COLS, SPLIT, BF16>, di->ordinal, (int)smem)) != cudaSuccess) return e;
+  decode_staged_kernel<KT, COLS, SPLIT, BF16><<<(unsigned)grid, SPLIT * COLS + 32, smem, stream>>>(a, tab, plan);
   count_launch();
   return cudaGetLastError();
 }
@@ -434,7 +447,7 @@ bool fits_256(const DecodeArgs& a) {
   const DeviceInfo* di = nullptr;
   if (current_device_info(&di) != cudaSuccess) return false;
   const int smem_sm = di->smem_per_sm;
-  return (int64_t)slots_off(a.W, a.K) + 2 * (int64_t)slot_bytes(a.W, KT, SPLIT, 256) + 1024 <= smem_sm;
+  return (int64_t)slots_off(a.W, a.K) + 2 * (int64_t)slot_bytes(a.W, KT, SPLIT, 256, a.bf16 ? 8 : 16) + 1024 <= smem_sm;
 }
 
 template <int KT, int SPLIT>
@@ -478,9 +491,11 @@ cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cu
 // the (K, W) pairs in which some alpha_j equals some beta_i (the row-copy case), stay on the other kernels.
 bool decode_staged_eligible(const DecodeArgs& a) {
   if (a.tune.kernel != 0 && a.tune.kernel != 3) return false;
-  const bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&
-                   a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
-  if (!(vec && a.C >= kStagedMinC)) return false;
+  bool vec = aligned16(a.Yt) && aligned16(a.Yh) && a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 &&
+             a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  // bfloat16: a column of four elements is 8 bytes, and every bulk copy must start and end on 16-byte boundaries
+  if (a.bf16) vec = vec && a.C % 8 == 0 && a.y_gs % 8 == 0 && a.y_rs % 8 == 0 && a.K <= kWholeMaxK;
+  if (!(vec && a.C >= kStagedMinC * (a.bf16 ? 2 : 1))) return false;
   for (int j = 0; j < a.K; ++j)
     for (int i = 0; i < a.W; ++i)
       if (nodes_coincide(a.K, a.W, j, i)) return false;
@@ -501,7 +516,8 @@ cudaError_t dispatch_whole(const DecodeArgs& a, const DecodeTables& tab, cudaStr
       const int64_t Cv = a.C / 4;
       const int64_t waste256 = (Cv + 255) / 256 * 256 - Cv, waste128 = (Cv + 127) / 128 * 128 - Cv;
       const bool want = a.tune.split == 1 || (a.tune.split == 0 && (a.tune.cols == 0 || a.tune.cols == 256) && waste256 <= waste128);
-      *taken = want && fits_256<KT, 1>(a);
+      *taken = (want || a.bf16) && fits_256<KT, 1>(a);
+      if (*taken && a.bf16) return launch_kt<KT, 256, 1, true>(a, tab, stream);
       return *taken ? launch_kt<KT, 256, 1>(a, tab, stream) : cudaSuccess;
     }
     return dispatch_whole<KT + 1>(a, tab, stream, taken);
@@ -512,6 +528,7 @@ cudaError_t launch_decode_staged(const DecodeArgs& a, const DecodeTables& tab, c
   bool taken = false;
   const cudaError_t e = dispatch_whole<>(a, tab, stream, &taken);
   if (taken) return e;
+  if (a.bf16) return cudaErrorInvalidConfiguration;  // (decode_staged_eligible admits bfloat16 only where the whole-row plan fits)
   if (a.tune.split == 4) return dispatch_kt<4>((a.K + 3) / 4, a, tab, stream);
   return dispatch_kt<2>((a.K + 1) / 2, a, tab, stream);
 }

@@ -97,6 +97,9 @@ DECODE_CASES = [
     (3, 7, 50, 36),        # coincident nodes
     (5, 9, 17, 33),        # odd length: element-wise path
     (32, 32, 5, 64),
+    (8, 12, 60, 128),      # the shortest rows the bulk-copy staged kernel takes with bfloat16 payloads
+    (16, 24, 9, 2056),     # several 256-column tiles per row and a ragged last one
+    (12, 20, 40, 1004),    # 1004 is not a multiple of 8: per-column kernel
 ]
 
 
