@@ -18,7 +18,8 @@ and the aggregate is reported.
 workload on the host cores.
 
 --case NAME times one kernel alone (tuning / profiling); --case grid prints the
-decoder's throughput over a grid of payload lengths on 3 GB problems.
+decoder's throughput over a grid of payload lengths on 3 GB problems, --case
+locategrid the locator over K in {8, 10, 12} x E in {1, 2, 3}.
 """
 from __future__ import annotations
 
@@ -372,6 +373,32 @@ def fma_peak(ap, dev):
             "note": "register-only loop, 16 independent chains per thread, 8 CTAs of 256 threads per SM; nominal = 148 SMs x 128 lanes x 2 x 1.965 GHz"}
 
 
+def locate_grid(ap, dev, G=65536, C=10):
+    """The locator over the paper's own grid (Section 4.2: K in {8, 10, 12}, E in {1, 2, 3}, no stragglers), linear
+    stand-in model, N(0, 10^2) noise on the E adversaries: ms per launch and groups/s."""
+    out = []
+    for K in (8, 10, 12):
+        for E in (1, 2, 3):
+            W = 2 * (K + E)
+            g = torch.Generator(device=dev)
+            g.manual_seed(1000 * K + E)
+            p = ap.make_params(K, W, E)
+            X = torch.rand((G, K, 64), generator=g, device=dev)
+            M = torch.randn((64, C), generator=g, device=dev) / 8.0
+            Yt = (ap.approxifer_encode(p, X) @ M).contiguous()
+            rng = np.random.Generator(np.random.PCG64(K * 10 + E))
+            bad = np.sort(rng.random((G, W)).argsort(axis=1)[:, :E], axis=1)
+            rows = torch.arange(G, device=dev)[:, None].expand(G, E)
+            Yt[rows, torch.as_tensor(bad, device=dev)] += torch.randn((G, E, C), generator=g, device=dev) * 10.0
+            mt = ap.mask_tensor(np.full(G, (1 << W) - 1, dtype=np.uint32), dev)
+            adv = torch.empty((G, E), dtype=torch.int32, device=dev)
+            trusted = torch.empty((G,), dtype=torch.int32, device=dev)
+            med, mn = time_launches(lambda: ap.approxifer_locate(p, Yt, mt, adv, trusted), 3, 10)
+            out.append({"K": K, "E": E, "W": W, "groups": G, "C": C, "ms": med, "ms_min": mn, "groups_per_s": G / med * 1e3,
+                        "located_equals_injected": float((adv.cpu().numpy() == bad).all(axis=1).mean())})
+    return out
+
+
 def host_cost(ap, dev):
     """Host time of one call (argument checks, plan, launch), from 1000 back-to-back calls on small problems."""
     out = []
@@ -540,6 +567,8 @@ def run_case(ap, dev, args):
         e = synthetic_decode(ap, dev, K, W, C, G, args.worker_major, iters, tuning)
         e.update(case="decode", dec_config=args.dec_config, wait_timeouts=ap.device_wait_timeouts())
         return e
+    if args.case == "locategrid":
+        return {"case": "locategrid", "locate": locate_grid(ap, dev)}
     if args.case == "fmapeak":
         return {"case": "fmapeak", **fma_peak(ap, dev)}
     if args.case == "hostcost":
@@ -551,12 +580,14 @@ def run_case(ap, dev, args):
     if op == "locateh":  # the locator with Algorithm 1's homogeneous system
         op, p = "locate", ap.make_params(w.K, w.W, w.E, 2)
     if op == "encode":
-        X = wl.queries(w, dev)
-        Xt = torch.empty((w.G, w.W, w.D), device=dev)
+        dt = torch.bfloat16 if args.bf16 else torch.float32
+        X = wl.queries(w, dev).to(dt)
+        Xt = torch.empty((w.G, w.W, w.D), device=dev, dtype=dt)
         if args.worker_major:
             Xt = Xt.view(w.W, w.G, w.D).permute(1, 0, 2)
-        med, mn = time_launches(lambda: ap.approxifer_encode(p, X, Xt), warm, iters)
-        nbytes = encode_bytes(w)
+        enc = ap.approxifer_encode_bf16 if args.bf16 else ap.approxifer_encode
+        med, mn = time_launches(lambda: enc(p, X, Xt), warm, iters)
+        nbytes = encode_bytes(w) // (2 if args.bf16 else 1)
     else:
         if cfg in (2, 3):
             Yt = wl.gaussian_predictions(w, dev)
@@ -648,10 +679,11 @@ def main():
     ap_.add_argument("--groups", type=int, default=None, help="override the number of groups (profiling only)")
     ap_.add_argument("--case", default=None,
                      choices=["decode2", "decode3", "decode4", "decode5", "locate5", "locateh5", "rational5", "pair5", "encode2", "encode3",
-                              "decode", "grid", "hostcost", "fmapeak"],
+                              "decode", "grid", "hostcost", "fmapeak", "locategrid"],
                      help="time one kernel alone (tuning / profiling) and print a short JSON line; `decode` takes --shape, "
                           "`grid` runs the decoder over payload lengths 10..256 on 3 GB problems")
     ap_.add_argument("--shape", default="8,12,64,1048576", help="K,W,C,G for --case decode")
+    ap_.add_argument("--bf16", action="store_true", help="--case encodeN: bfloat16 payloads")
     ap_.add_argument("--worker-major", action="store_true", help="--case: coded rows stored [W][G][*] (one batch per worker)")
     ap_.add_argument("--dec-config", default=None, help="kernel,stages,ctas_per_sm,cols,split for the decoder (--case, tuning)")
     args = ap_.parse_args()
@@ -786,6 +818,7 @@ def main():
     if not args.no_others and world == 1 and args.groups is None:
         line["others"] = other_workloads(ap, dev, peak)
         line["decode_grid_3GB"] = decode_grid(ap, dev)
+        line["locate_grid"] = locate_grid(ap, dev)
         line["host_cost"] = host_cost(ap, dev)
         line["fma_peak"] = fma_peak(ap, dev)
     line.update({

@@ -170,6 +170,28 @@ struct PayloadBf16x4 {
   }
   static __device__ __forceinline__ void store(Store* p, Vec v) { __stcs(p, make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w))); }
 };
+// eight bfloat16 elements as one 16-byte column (the encoder's choice when alignment and K allow: twice the bytes
+// in flight per thread of the 8-byte path)
+struct float8 {
+  float4 lo, hi;
+};
+struct PayloadBf16x8 {
+  using Store = uint4;
+  using Vec = float8;
+  static constexpr int kLanes = 8, kElemBytes = 2;
+  static __device__ __forceinline__ Vec load(const Store* p) {
+    const uint4 u = __ldcs(p);
+    Vec v;
+    v.lo = make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u), __uint_as_float(u.y << 16),
+                       __uint_as_float(u.y & 0xffff0000u));
+    v.hi = make_float4(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xffff0000u), __uint_as_float(u.w << 16),
+                       __uint_as_float(u.w & 0xffff0000u));
+    return v;
+  }
+  static __device__ __forceinline__ void store(Store* p, Vec v) {
+    __stcs(p, make_uint4(pack_bf16x2(v.lo.x, v.lo.y), pack_bf16x2(v.lo.z, v.lo.w), pack_bf16x2(v.hi.x, v.hi.y), pack_bf16x2(v.hi.z, v.hi.w)));
+  }
+};
 struct PayloadBf16 {
   using Store = unsigned short;
   using Vec = float;

@@ -29,6 +29,20 @@ struct VecOps<float4> {
   }
 };
 template <>
+struct VecOps<float8> {
+  static constexpr int kLanes = 8;
+  static __device__ __forceinline__ float8 mul(float w, float8 x) {
+    float8 r;
+    r.lo = VecOps<float4>::mul(w, x.lo), r.hi = VecOps<float4>::mul(w, x.hi);
+    return r;
+  }
+  static __device__ __forceinline__ float8 fma(float w, float8 x, float8 a) {
+    float8 r;
+    r.lo = VecOps<float4>::fma(w, x.lo, a.lo), r.hi = VecOps<float4>::fma(w, x.hi, a.hi);
+    return r;
+  }
+};
+template <>
 struct VecOps<float> {
   static constexpr int kLanes = 1;
   static __device__ __forceinline__ float mul(float w, float x) { return w * x; }
@@ -81,7 +95,7 @@ cudaError_t launch_one(const EncodeArgs& a, const EncodeTables& tab, cudaStream_
   // size: each CTA then reads and writes whole contiguous pieces of K and W rows, which HBM serves slightly
   // better (+0.8 % on workload 2) than the 4 KB pieces of 256-thread CTAs.
   // (K <= 16: beyond that 768 threads do not leave a thread enough registers for its K inputs)
-  if constexpr (P::kLanes == 4 && K <= 16) {
+  if constexpr (P::kLanes == 4 && K <= 16) {  // (16-byte columns of fp32, 8-byte columns of bfloat16)
     if (Dv % kEncodeWideThreads == 0) {
       const int64_t blocks = items / kEncodeWideThreads;
       if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
@@ -139,7 +153,9 @@ cudaError_t launch_encode(const EncodeArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   const EncodeTables& tab = encode_tables(a.K, a.W);
   const bool by4 = a.D % 4 == 0 && a.x_gs % 4 == 0 && a.x_rs % 4 == 0 && a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
-  if (a.bf16) {  // four bfloat16 elements are one 8-byte column
+  if (a.bf16) {  // eight bfloat16 elements are one 16-byte column (K <= 16: a thread keeps 8 K inputs), four an 8-byte one
+    const bool by8 = a.D % 8 == 0 && a.x_gs % 8 == 0 && a.x_rs % 8 == 0 && a.o_gs % 8 == 0 && a.o_rs % 8 == 0;
+    if (by8 && a.K <= 16 && aligned16(a.X) && aligned16(a.Xt)) return dispatch_k<PayloadBf16x8>(a, tab, stream);
     if (by4 && aligned8(a.X) && aligned8(a.Xt)) return dispatch_k<PayloadBf16x4>(a, tab, stream);
     return dispatch_k<PayloadBf16>(a, tab, stream);
   }
