@@ -344,14 +344,35 @@ __global__ void __launch_bounds__(kRowsThreads, M > 10 ? 2 : 3) locate_rows_kern
       for (int i = 0; i < n; i += 2) {  // an odd n reads one padded (zero) entry
         const double2 nn = *reinterpret_cast<const double2*>(nr + i);
         const double u0 = nn.x * (double)ysm[i * kRowsThreads], u1 = nn.y * (double)ysm[(i + 1) * kRowsThreads];
+        if constexpr (M >= 14) {
+          // The largest factors leave no registers to spare and spill; there the powers b_i^l are rebuilt on the
+          // way (the same products in the same order as the table holds, so the same values) instead of being
+          // loaded: one multiplication per power against five 128-bit shared-memory loads per worker, each of
+          // which costs one pass per group that the warp's threads belong to.  Measured on 65,536 groups of 10
+          // classes: K+E = 14: 1.87 -> 1.50 ms, 15: 2.99 -> 2.59 ms; for K+E <= 13 the table is as fast or faster.
+          const double2 bb = *reinterpret_cast<const double2*>(&sm.xs[i]);
+          double p0 = bb.x, p1 = bb.y;
+          row[0] = fma(u0, 1.0, row[0]);
+          row[0] = fma(u1, 1.0, row[0]);
 #pragma unroll
-        for (int l = 0; l < MP; l += 2) {
-          const double2 p0 = *reinterpret_cast<const double2*>(&sm.pw[i][l]);
-          const double2 p1 = *reinterpret_cast<const double2*>(&sm.pw[i + 1][l]);
-          row[l] = fma(u0, p0.x, row[l]);
-          row[l + 1] = fma(u0, p0.y, row[l + 1]);
-          row[l] = fma(u1, p1.x, row[l]);
-          row[l + 1] = fma(u1, p1.y, row[l + 1]);
+          for (int l = 1; l < M; ++l) {
+            row[l] = fma(u0, p0, row[l]);
+            row[l] = fma(u1, p1, row[l]);
+            if (l + 1 < M) {
+              p0 *= bb.x;
+              p1 *= bb.y;
+            }
+          }
+        } else {
+#pragma unroll
+          for (int l = 0; l < MP; l += 2) {
+            const double2 p0 = *reinterpret_cast<const double2*>(&sm.pw[i][l]);
+            const double2 p1 = *reinterpret_cast<const double2*>(&sm.pw[i + 1][l]);
+            row[l] = fma(u0, p0.x, row[l]);
+            row[l + 1] = fma(u0, p0.y, row[l + 1]);
+            row[l] = fma(u1, p1.x, row[l]);
+            row[l + 1] = fma(u1, p1.y, row[l + 1]);
+          }
         }
       }
       // fold the equation  sum_k row[k+1] q_k = -row[0]  (weight w, 1 at the start) into (D, U, d): the
