@@ -612,6 +612,8 @@ def run_case(ap, dev, args):
             nbytes = locate_bytes(w, m) + 4 * w.G * w.K * w.C
         elif op == "pair":
             Yh = torch.empty((w.G, w.K, w.C), device=dev)
+            if args.one_pass is not None:  # 1: the one-pass kernel, 0: the two launches; default: the library's choice
+                p = ap.make_params(w.K, w.W, w.E, 4 if args.one_pass else 8)
             med, mn = time_launches(lambda: ap.approxifer_locate_decode(p, Yt, mt, Yh), warm, iters)
             nbytes = locate_bytes(w, m) + 4 * w.G * w.K * w.C
         else:
@@ -683,6 +685,7 @@ def main():
                      help="time one kernel alone (tuning / profiling) and print a short JSON line; `decode` takes --shape, "
                           "`grid` runs the decoder over payload lengths 10..256 on 3 GB problems")
     ap_.add_argument("--shape", default="8,12,64,1048576", help="K,W,C,G for --case decode")
+    ap_.add_argument("--one-pass", type=int, default=None, help="--case pair5: 1 forces the one-pass kernel, 0 the two launches")
     ap_.add_argument("--bf16", action="store_true", help="--case encodeN: bfloat16 payloads")
     ap_.add_argument("--worker-major", action="store_true", help="--case: coded rows stored [W][G][*] (one batch per worker)")
     ap_.add_argument("--dec-config", default=None, help="kernel,stages,ctas_per_sm,cols,split for the decoder (--case, tuning)")

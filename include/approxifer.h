@@ -66,6 +66,8 @@ extern "C" {
 #define APPROXIFER_SIGN_RANK 0u         /* decoder sign (-1)^(rank of worker i among those used); default */
 #define APPROXIFER_SIGN_WORKER_INDEX 1u /* decoder sign (-1)^i, the decoding equation read literally */
 #define APPROXIFER_LOCATE_HOMOGENEOUS 2u /* locator: Algorithm 1's homogeneous system (|Q| = 1) instead of Q_0 = 1 */
+#define APPROXIFER_ONE_PASS 4u           /* approxifer_locate_decode: one kernel for both steps wherever it exists */
+#define APPROXIFER_TWO_LAUNCHES 8u       /* approxifer_locate_decode: always the two kernels back to back */
 
 /* status[g] bits */
 #define APPROXIFER_ST_NO_WORKERS 1u             /* decode: no worker present; the group's output is zero-filled */
@@ -203,11 +205,20 @@ int approxifer_decode_rational(const approxifer_params* params, int64_t G, int64
 /*
  * The decoder's two steps in one call (Section 3, "ApproxIFER Decoding", steps 1 and 2): locate the E
  * Byzantine workers of every group (Algorithm 2), then decode from the workers that are present and were
- * not located.  Equivalent to approxifer_locate followed by approxifer_decode with `trusted_mask` as the
- * mask, enqueued back to back on `cuda_stream`.  `trusted_mask` [G] is required (it carries the result of
- * step 1 to step 2 on the device); `adv` [G][E], `n_used` [G], `locate_status` [G] and `decode_status` [G]
- * are as in the two entry points (`adv` is required, the other three may be NULL).
+ * not located.  Equivalent, bit for bit, to approxifer_locate followed by approxifer_decode with
+ * `trusted_mask` as the mask.  `trusted_mask` [G] is required (it carries the result of step 1 to step 2 on the
+ * device); `adv` [G][E], `n_used` [G], `locate_status` [G] and `decode_status` [G] are as in the two entry
+ * points (`adv` is required, the other three may be NULL).
+ *
+ * The call is either one kernel -- the locator with the decoding as its tail, available for Algorithm 2's form
+ * with K+E <= 10 and C <= 128 -- or the two kernels back to back on `cuda_stream`.  One kernel saves a launch
+ * and a pass over the predictions, but decodes at the locator's low occupancy: it wins on small batches
+ * (K = 8, W = 24, E = 2, C = 10: 44 us against 52 us up to 1,024 groups, equal at 4,096) and loses about a tenth
+ * on large ones (641 us against 591 us at 65,536 groups), so by default it is taken for batches of up to
+ * APPROXIFER_ONE_PASS_MAX_GROUPS groups.  APPROXIFER_ONE_PASS / APPROXIFER_TWO_LAUNCHES in params.flags override
+ * the choice (ONE_PASS where no such kernel exists still runs the two).
  */
+#define APPROXIFER_ONE_PASS_MAX_GROUPS 4096
 int approxifer_locate_decode(const approxifer_params* params, int64_t G, int64_t C,
                              const float* Yt, int64_t yt_gstride, int64_t yt_rstride,
                              const uint32_t* mask,

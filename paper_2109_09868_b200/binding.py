@@ -22,6 +22,7 @@ E_NULL, E_RANGE, E_PARAM, E_CUDA, E_WORKSPACE, E_TOO_LARGE = -1, -2, -3, -4, -5,
 STATIC_WORKSPACE_BYTES = 32 << 20
 SIGN_RANK, SIGN_WORKER_INDEX = 0, 1
 LOCATE_HOMOGENEOUS = 2
+ONE_PASS, TWO_LAUNCHES = 4, 8
 ST_NO_WORKERS, ST_FEW_WORKERS, ST_LOCATE_UNDERDETERMINED, ST_NONFINITE, ST_TIMEOUT = 1, 2, 4, 8, 16
 
 EXPORTS = (

@@ -38,7 +38,8 @@ namespace {
 int check_kw(const approxifer_params* p) {
   if (p == nullptr) return APPROXIFER_E_NULL;
   if (p->K < 1 || p->K > APPROXIFER_MAX_K || p->W < 2 || p->W > APPROXIFER_MAX_W) return APPROXIFER_E_RANGE;
-  if (p->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS)) return APPROXIFER_E_PARAM;
+  if (p->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS | APPROXIFER_ONE_PASS | APPROXIFER_TWO_LAUNCHES))
+    return APPROXIFER_E_PARAM;
   return APPROXIFER_OK;
 }
 
@@ -203,6 +204,20 @@ int approxifer_locate_decode(const approxifer_params* params, int64_t G, int64_t
   if (rc) return rc;
   if ((rc = check_layout(G, C, yh_rstride))) return rc;
   if (yh_gstride < 0) return APPROXIFER_E_RANGE;
+  // one pass where the thread-per-class locator can carry the decoding as its tail (all classes of a group in one
+  // CTA, a small factor), else the two kernels back to back; the results are bit-identical
+  if (params->E >= 1 && 2 * (params->K + params->E) <= params->W && yt_gstride >= 0 && G > 0 && Yt != nullptr && mask != nullptr &&
+      adv != nullptr && trusted_mask != nullptr && check_layout(G, C, yt_rstride) == APPROXIFER_OK) {
+    LocateArgs a{Yt, mask, adv, trusted_mask, locate_status, yt_gstride, yt_rstride, G, C, params->K, params->W, params->E, params->flags};
+    const bool want = (params->flags & APPROXIFER_TWO_LAUNCHES) ? false
+                      : (params->flags & APPROXIFER_ONE_PASS)   ? true
+                                                                : G <= APPROXIFER_ONE_PASS_MAX_GROUPS;
+    if (want && locate_fuse_eligible(a)) {
+      a.Yh = Yhat, a.o_gs = yh_gstride, a.o_rs = yh_rstride;
+      a.fuse_decode = 1, a.n_used = n_used, a.decode_status = decode_status;
+      return from_cuda(launch_locate(a, static_cast<cudaStream_t>(cuda_stream)));
+    }
+  }
   rc = approxifer_locate(params, G, C, Yt, yt_gstride, yt_rstride, mask, adv, trusted_mask, locate_status, cuda_stream);
   if (rc) return rc;
   return approxifer_decode(params, G, C, Yt, yt_gstride, yt_rstride, trusted_mask, Yhat, yh_gstride, yh_rstride, n_used,

@@ -70,6 +70,10 @@ struct LocateArgs {
   float* Yh = nullptr;
   int64_t o_gs = 0, o_rs = 0;
   int32_t force_warp_kernel = 0;  // test hook: the warp-per-group kernel also where the thread-per-class one would run
+  // locate and decode in one pass (Yh, o_gs, o_rs above receive the decoded predictions instead of Algorithm 3's)
+  int32_t fuse_decode = 0;
+  int32_t* n_used = nullptr;          // decode's optional outputs
+  uint32_t* decode_status = nullptr;
 };
 
 // Each returns a cudaError_t from the launch (cudaSuccess if nothing to do).
@@ -100,6 +104,10 @@ cudaError_t launch_decode_small(const DecodeArgs& a, const DecodeTables& tab, cu
 constexpr int kLocateRowsMaxM = 15;
 // ... and its alternative last steps (Algorithm 1's homogeneous system, Algorithm 3) for K+E <= kLocateAltMaxM
 constexpr int kLocateAltMaxM = 13;
+// ... and the one-pass locate + decode for K+E <= kLocateFuseMaxM and at most kLocateFuseMaxC classes
+constexpr int kLocateFuseMaxM = 10;
+constexpr int kLocateFuseMaxC = 128;
+bool locate_fuse_eligible(const LocateArgs& a);
 cudaError_t launch_locate_rows(const LocateArgs& a, const LocateTables& tab, cudaStream_t stream);
 
 void count_launch(int n = 1);

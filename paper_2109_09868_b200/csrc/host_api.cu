@@ -96,7 +96,7 @@ int approxifer_decode_host(const approxifer_params* params, int64_t G, int64_t C
                            void* const* cuda_streams, int n_streams) {
   if (params == nullptr) return APPROXIFER_E_NULL;
   if (params->K < 1 || params->K > APPROXIFER_MAX_K || params->W < 2 || params->W > APPROXIFER_MAX_W) return APPROXIFER_E_RANGE;
-  if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS)) return APPROXIFER_E_PARAM;
+  if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS | APPROXIFER_ONE_PASS | APPROXIFER_TWO_LAUNCHES)) return APPROXIFER_E_PARAM;
   if (G < 0 || C < 1 || C > (int64_t(1) << 31)) return APPROXIFER_E_RANGE;
   if (G == 0) return APPROXIFER_OK;
   if (hYt == nullptr || hmask == nullptr || hYhat == nullptr || workspace == nullptr || cuda_streams == nullptr)
@@ -153,7 +153,7 @@ int approxifer_locate_host(const approxifer_params* params, int64_t G, int64_t C
   if (params->K < 1 || params->K > APPROXIFER_MAX_K || params->W < 2 || params->W > APPROXIFER_MAX_W || params->E < 0)
     return APPROXIFER_E_RANGE;
   if (params->E < 1 || 2 * (params->K + params->E) > params->W) return APPROXIFER_E_PARAM;
-  if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS)) return APPROXIFER_E_PARAM;
+  if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS | APPROXIFER_ONE_PASS | APPROXIFER_TWO_LAUNCHES)) return APPROXIFER_E_PARAM;
   if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateAltMaxM) return APPROXIFER_E_PARAM;
   if (G < 0 || C < 1 || C > (int64_t(1) << 31)) return APPROXIFER_E_RANGE;
   if (G == 0) return APPROXIFER_OK;

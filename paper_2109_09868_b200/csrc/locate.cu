@@ -267,12 +267,18 @@ cudaError_t dispatch_m(int m, const LocateArgs& a, const LocateTables& tab, cuda
 
 }  // namespace
 
+// Locate and decode in one pass: Algorithm 2's form of the per-class step, a thread per (group, class) with all
+// classes of a group in one CTA, and a factor small enough to leave the decoding tail its registers.
+bool locate_fuse_eligible(const LocateArgs& a) {
+  return !(a.flags & kFlagLocateHomogeneous) && a.K + a.E <= kLocateFuseMaxM && a.C <= kLocateFuseMaxC;
+}
+
 cudaError_t launch_locate(const LocateArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   const LocateTables& tab = locate_tables(a.K, a.W);
   const int m = a.K + a.E;
   // (the homogeneous form and Algorithm 3 exist in the thread-per-class kernel only; the entry points have checked K+E)
-  const bool alt = (a.flags & kFlagLocateHomogeneous) || a.Yh != nullptr;
+  const bool alt = (a.flags & kFlagLocateHomogeneous) || a.Yh != nullptr;  // (the fused pass is one of them: api.cu has checked its range)
   if (alt ? m <= kLocateAltMaxM : (m <= kLocateRowsMaxM && !a.force_warp_kernel))
     return launch_locate_rows(a, tab, stream);
   if (a.W <= 8) return dispatch_m<8>(m, a, tab, stream);

@@ -28,7 +28,7 @@ namespace {
 
 using namespace locate_detail;
 
-static_assert(sizeof(LocateArgs) + sizeof(LocateTables) + sizeof(LocateBasis) + 16 <= 32764,
+static_assert(sizeof(LocateArgs) + sizeof(LocateTables) + sizeof(LocateBasis) + sizeof(DecodeTables) + 16 <= 32764,
               "locator kernel parameters exceed the launch limit (blocks above 4 KB need CUDA 12.1 or later)");
 
 constexpr int kRowsThreads = 128;
@@ -238,12 +238,16 @@ __device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double 
 // sense with |Q| = 1; basis, rows, selection and vote are shared.  MODE 2: Algorithm 3 -- the same per-class
 // solve as mode 0, then no selection and no vote: P is recovered and r = P/Q is evaluated at the K nodes alpha_j
 // (a decoder that absorbs up to E wrong predictions instead of locating them).
-constexpr int kModeLocate = 0, kModeHomogeneous = 1, kModeRational = 2;
+// MODE 3: mode 0 followed, in the same launch, by the decoding of every group from the workers that are present and
+// were not located (Section 3, "ApproxIFER Decoding", steps 1 and 2 in one pass): the same terms in the same order
+// as the decoder kernels, so the result is bit-identical to the two launches.
+constexpr int kModeLocate = 0, kModeHomogeneous = 1, kModeRational = 2, kModeLocateDecode = 3;
 
 template <int NMAX, int M, int MODE>
 __global__ void __launch_bounds__(kRowsThreads, M > 10 ? 2 : 3) locate_rows_kernel(const __grid_constant__ LocateArgs a,
                                                                       const __grid_constant__ LocateTables tab,
                                                                       const __grid_constant__ LocateBasis basis,
+                                                                      const __grid_constant__ DecodeTables dtab,
                                                                       const int gpb) {
   using SM = GroupSmem<NMAX, M>;
   constexpr int MP = SM::MP;
@@ -548,13 +552,14 @@ __global__ void __launch_bounds__(kRowsThreads, M > 10 ? 2 : 3) locate_rows_kern
   }
   // ---- the E most voted workers of each group, ties to the lower index; lane = rank ----------------
   for (int s = warp; s < ng; s += kRowsWarps) {
-    const SM& sm = groups[s];
+    SM& sm = groups[s];
     const int64_t g = g_first + s;
     const uint32_t mask = sm.mask;
     if (sm.n < 0) {
       for (int e = lane; e < E; e += 32) a.adv[g * E + e] = -1;
       if (lane == 0) {
         a.trusted[g] = mask;
+        sm.pad = (int)mask;  // (kept for the decoding tail)
         if (a.status) a.status[g] = sm.status;
       }
       continue;
@@ -577,7 +582,62 @@ __global__ void __launch_bounds__(kRowsThreads, M > 10 ? 2 : 3) locate_rows_kern
     if (elected) a.adv[g * E + __popc(picked & ((1u << lane) - 1u))] = my_worker;
     if (lane == 0) {
       a.trusted[g] = mask & ~wbits;
+      sm.pad = (int)(mask & ~wbits);
       if (a.status) a.status[g] = sm.status;
+    }
+  }
+
+  if constexpr (MODE == kModeLocateDecode) {
+    // ---- decoding from the trusted workers, one thread per (group, class) again ----------------------
+    // Yhat[g][j][c] = sum_i s_i rg_ij y_ic / sum_i s_i rg_ij over the trusted workers i in ascending order,
+    // rg_ij = 1/(alpha_j - beta_i): the decoder kernels' terms, order and roundings.  The predictions come
+    // back from global memory (L2: this CTA has just read them); the table sits where the threads' prediction
+    // columns were.
+    constexpr int KMAX = M - 1;  // K = M - E, E >= 1
+    __syncthreads();  // the trusted masks are in shared memory, the prediction columns are dead
+    float* rgs = reinterpret_cast<float*>(scratch);
+    const int K = a.K, W = a.W;
+    for (int idx = tid; idx < W * K; idx += kRowsThreads) rgs[idx] = dtab.rg[idx];
+    __syncthreads();
+    const bool literal = (a.flags & kFlagSignWorkerIndex) != 0;
+    for (int64_t t = tid; t < n_tasks; t += kRowsThreads) {
+      const int s = (int)(t / a.C);
+      const int64_t c = t - (int64_t)s * a.C;
+      const int64_t g = g_first + s;
+      const uint32_t trusted = (uint32_t)groups[s].pad;
+      const float* Yc = a.Yt + g * a.y_gs + c;
+      float acc[KMAX], den[KMAX];
+#pragma unroll
+      for (int j = 0; j < KMAX; ++j) acc[j] = den[j] = 0.f;
+      int r = 0;
+      for (uint32_t m = trusted; m; m &= m - 1, ++r) {
+        const int i = __ffs((int)m) - 1;
+        const float y = __ldg(Yc + (int64_t)i * a.y_rs);
+        const uint32_t odd = ((literal ? (uint32_t)i : (uint32_t)r) & 1u) << 31;
+#pragma unroll
+        for (int j = 0; j < KMAX; ++j) {
+          if (j < K) {
+            const float w = __uint_as_float(__float_as_uint(rgs[i * K + j]) ^ odd);
+            acc[j] = fmaf(w, y, acc[j]);
+            den[j] = __fadd_rn(den[j], w);
+          }
+        }
+      }
+      const int n = r;
+#pragma unroll
+      for (int j = 0; j < KMAX; ++j) {
+        if (j < K) {
+          const int cq = dtab.any_coin ? (int)dtab.coin[j] : -1;  // alpha_j == beta_cq: the interpolant takes that value
+          float v = acc[j] * __frcp_rn(den[j]);
+          if (cq >= 0 && ((trusted >> cq) & 1u)) v = __ldg(Yc + (int64_t)cq * a.y_rs);
+          if (n == 0) v = 0.f;
+          a.Yh[g * a.o_gs + (int64_t)j * a.o_rs + c] = v;
+        }
+      }
+      if (c == 0) {
+        if (a.n_used) a.n_used[g] = n;
+        if (a.decode_status) a.decode_status[g] = (n == 0 ? kStNoWorkers : 0u) | (n < K ? kStFewWorkers : 0u);
+      }
     }
   }
 }
@@ -588,7 +648,7 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
   int64_t gpb = a.C >= kRowsThreads ? 1 : kRowsThreads / a.C;
   if (gpb > kMaxGroupsPerCta) gpb = kMaxGroupsPerCta;
   // per group: its block, and for Algorithm 3 the M x M table that carries P to the alpha nodes
-  const size_t per_group = sizeof(GroupSmem<NMAX, M>) + (a.Yh != nullptr ? (size_t)M * M * sizeof(double) : 0);
+  const size_t per_group = sizeof(GroupSmem<NMAX, M>) + ((a.Yh != nullptr && !a.fuse_decode) ? (size_t)M * M * sizeof(double) : 0);
   // per-thread predictions, aliased with the set-up scratch (the warps' reflectors and the transposed full-set basis)
   const size_t y_bytes = scratch_bytes<NMAX, M>();
   // shared memory for three CTAs per SM (K+E <= 10: 168 registers per thread) or two (the larger factors
@@ -608,10 +668,15 @@ cudaError_t launch_rows_nm(const LocateArgs& a, const LocateTables& tab, cudaStr
       struct Tag {};
       if ((e = ensure_dynamic_smem<Tag>(locate_rows_kernel<NMAX, M, MODE>, di->ordinal, (int)smem)) != cudaSuccess) return e;
     }
-    locate_rows_kernel<NMAX, M, MODE><<<(unsigned)blocks, kRowsThreads, smem, stream>>>(a, tab, locate_basis(a.W, M), (int)gpb);
+    locate_rows_kernel<NMAX, M, MODE><<<(unsigned)blocks, kRowsThreads, smem, stream>>>(a, tab, locate_basis(a.W, M),
+                                                                                        decode_tables(a.K, a.W), (int)gpb);
     count_launch();
     return cudaGetLastError();
   };
+  if constexpr (M <= kLocateFuseMaxM) {
+    if (a.fuse_decode) return run(std::integral_constant<int, kModeLocateDecode>{});
+  }
+  if (a.fuse_decode) return cudaErrorInvalidConfiguration;
   if constexpr (M <= kLocateAltMaxM) {
     if (a.Yh != nullptr) return run(std::integral_constant<int, kModeRational>{});
     if (a.flags & kFlagLocateHomogeneous) return run(std::integral_constant<int, kModeHomogeneous>{});

@@ -56,7 +56,7 @@ extern "C" int approxifer_encode_host_static(const approxifer_params* params, in
                                              float* hXt, void* cuda_stream) {
   if (params == nullptr) return APPROXIFER_E_NULL;
   if (params->K < 1 || params->K > APPROXIFER_MAX_K || params->W < 2 || params->W > APPROXIFER_MAX_W) return APPROXIFER_E_RANGE;
-  if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS)) return APPROXIFER_E_PARAM;
+  if (params->flags & ~(APPROXIFER_SIGN_WORKER_INDEX | APPROXIFER_LOCATE_HOMOGENEOUS | APPROXIFER_ONE_PASS | APPROXIFER_TWO_LAUNCHES)) return APPROXIFER_E_PARAM;
   if (G < 0 || D < 1 || D > (int64_t(1) << 31)) return APPROXIFER_E_RANGE;
   if (G == 0) return APPROXIFER_OK;
   if (hX == nullptr || hXt == nullptr) return APPROXIFER_E_NULL;

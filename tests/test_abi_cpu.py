@@ -56,7 +56,7 @@ def test_encode_argument_errors_are_reported_on_the_host():
     assert _encode_rc(4, 5, 1, 8, orr=4) == binding.E_RANGE
     assert _encode_rc(4, 5, 1, 8, x=None) == binding.E_NULL
     assert _encode_rc(4, 5, 1, 8, xt=None) == binding.E_NULL
-    assert _encode_rc(4, 5, 1, 8, flags=4) == binding.E_PARAM  # unknown flag bit
+    assert _encode_rc(4, 5, 1, 8, flags=16) == binding.E_PARAM  # unknown flag bit
     assert _encode_rc(4, 5, 0, 8, x=None, xt=None) == binding.OK  # G = 0: valid no-op
     assert ap.load().approxifer_encode(None, 1, 8, 1, 32, 8, 1, 40, 8, None) == binding.E_NULL
 
@@ -86,7 +86,7 @@ def test_flags_each_entry_point_ignores_or_rejects():
     lib = ap.load()
     both = binding.SIGN_WORKER_INDEX | binding.LOCATE_HOMOGENEOUS
     q = ap.make_params(8, 24, 2, both)
-    bad = ap.make_params(8, 24, 2, 4)
+    bad = ap.make_params(8, 24, 2, 16)
     assert lib.approxifer_encode(ctypes.byref(q), 0, 8, None, 64, 8, None, 192, 8, None) == binding.OK
     assert lib.approxifer_encode(ctypes.byref(bad), 0, 8, None, 64, 8, None, 192, 8, None) == binding.E_PARAM
     assert lib.approxifer_decode(ctypes.byref(q), 0, 10, None, 240, 10, None, None, 80, 10, None, None, None) == binding.OK

@@ -605,6 +605,44 @@ def test_locate_decode_in_one_call_equals_the_two_steps():
     assert int(lst[7]) == 4 and int(n_used[7]) == 10
 
 
+@pytest.mark.parametrize("K,E,S,W,C,G,flags", [(8, 2, 2, 24, 10, 257, 0),     # one pass: a thread per (group, class)
+                                               (8, 2, 0, 20, 10, 100, 1),     # ... with the literal sign rule
+                                               (1, 1, 0, 5, 10, 60, 0),       # ... alpha_0 = beta_2: a copied row
+                                               (4, 1, 2, 12, 128, 40, 0),     # ... the most classes the one-pass kernel takes
+                                               (4, 1, 2, 12, 129, 40, 0),     # one class more: two launches
+                                               (9, 2, 1, 23, 10, 90, 0)])     # K+E = 11: two launches
+def test_locate_decode_one_pass_and_two_launches_agree_with_the_two_steps(K, E, S, W, C, G, flags):
+    """approxifer_locate_decode runs as one kernel where the thread-per-class locator can carry the decoding as
+    its tail, else as two launches; either way the located sets, trusted masks, decoded values (bit for bit),
+    worker counts and status words equal those of approxifer_locate followed by approxifer_decode."""
+    Yt, mask, truth = linear_case(K, W, E, S, G, C, seed=K * 100 + C)
+    mask[3] = (1 << (2 * (K + E) - 1)) - 1  # one worker short of 2(K+E): nothing located, decoded from all present
+    mask[5] = 0                             # nobody answered
+    p = ap.make_params(K, W, E, flags | binding.ONE_PASS)
+    Yd, md = Yt.to(dev()), ap.mask_tensor(mask)
+    n_used = torch.empty(G, dtype=torch.int32, device=dev())
+    lst = torch.empty(G, dtype=torch.int32, device=dev())
+    dst = torch.empty(G, dtype=torch.int32, device=dev())
+    out = torch.full((G, K, C + 3), CANARY, device=dev())  # padded rows: element strides, canaries behind every row
+    Yh, adv, trusted = ap.approxifer_locate_decode(p, Yd, md, Yhat=out[:, :, :C], n_used=n_used, locate_status=lst, decode_status=dst)
+    lst2 = torch.empty(G, dtype=torch.int32, device=dev())
+    adv2, trusted2 = ap.approxifer_locate(p, Yd, md, status=lst2)
+    n2 = torch.empty(G, dtype=torch.int32, device=dev())
+    dst2 = torch.empty(G, dtype=torch.int32, device=dev())
+    Yh2 = ap.approxifer_decode(p, Yd, trusted2, n_used=n2, status=dst2, tuning=ap.decode_tuning(kernel=1))
+    assert torch.equal(adv, adv2) and torch.equal(trusted, trusted2) and torch.equal(lst, lst2)
+    assert torch.equal(Yh.contiguous().view(torch.int32), Yh2.view(torch.int32))
+    assert torch.equal(n_used, n2) and torch.equal(dst, dst2)
+    assert bool((out[:, :, C:] == CANARY).all())
+    if flags == 0:
+        ref = oracle.locate(K, W, E, Yt.numpy(), mask)
+        solid = (ref["min_gap"] > 1.0 + 1e-6) & (ref["vote_margin"] > 0) & ((ref["status"] & oracle.ST_ORACLE_RANK_DEFICIENT) == 0)
+        solid |= (ref["status"] & oracle.ST_LOCATE_UNDERDETERMINED) != 0
+        np.testing.assert_array_equal(adv.cpu().numpy()[solid], ref["adv"][solid])
+        check_decode(K, W, Yt, trusted.cpu().numpy().view(np.uint32), Yh, n_used, dst)
+    assert int(lst[3]) == 4 and int(n_used[3]) == 2 * (K + E) - 1 and int(dst[5]) & 1
+
+
 # ------------------------------------------------------------------ randomized shapes
 
 @pytest.mark.parametrize("seed", range(24))
