@@ -453,7 +453,12 @@ def other_workloads(ap, dev, peak):
     Xt_wm = Xt.view(w2.W, G2, w2.D).permute(1, 0, 2)
     med, mn = time_launches(lambda: ap.approxifer_encode(p2, X, Xt_wm), 3, 20)
     entry("configs[1] encode, coded queries written worker-major [W][G][D]", encode_bytes(w2g), med, mn, G2)
-    del X, Xt, Xt_wm
+    del Xt, Xt_wm
+    # ... and scattered: every worker's batch a buffer of its own (the layout of peer-resident batches)
+    rows = [torch.empty((G2, w2.D), device=dev) for _ in range(w2.W)]
+    med, mn = time_launches(lambda: ap.approxifer_encode_scatter(p2, X, rows), 3, 20)
+    entry("configs[1] encode, coded queries scattered to one buffer per worker (approxifer_encode_scatter)", encode_bytes(w2g), med, mn, G2)
+    del X, rows
     Yt = wl.gaussian_predictions(w2, dev)
     m2 = wl.masks(w2)
     mt = ap.mask_tensor(m2, dev)
@@ -506,8 +511,14 @@ def other_workloads(ap, dev, peak):
     entry("configs[4] decode from trusted K=8 W=24 C=10 (L2-resident)", decode_bytes(w5, t5), med, mn, w5.G)
     med, mn = time_launches(lambda: ap.approxifer_decode(p5, Yt_wm, trusted, Yh), 3, 10)
     entry("configs[4] decode from trusted, predictions stored worker-major [W][G][C]", decode_bytes(w5, t5), med, mn, w5.G)
+    rows5 = [Yt[:, i].contiguous() for i in range(w5.W)]
+    med, mn = time_launches(lambda: ap.approxifer_locate_gather(p5, rows5, mt), 3, 10)
+    entry("configs[4] locate, predictions gathered from one buffer per worker (approxifer_locate_gather)", locate_bytes(w5, m5), med, mn, w5.G)
+    med, mn = time_launches(lambda: ap.approxifer_decode_gather(p5, rows5, trusted, Yh), 3, 10)
+    entry("configs[4] decode from trusted, gathered from one buffer per worker (approxifer_decode_gather)", decode_bytes(w5, t5), med, mn, w5.G)
+    del rows5
     med, mn = time_launches(lambda: ap.approxifer_locate_decode(p5, Yt, mt, Yh), 3, 10)
-    entry("configs[4] locate + decode from trusted through approxifer_locate_decode (two launches)",
+    entry("configs[4] locate + decode from trusted through approxifer_locate_decode (two launches at this size)",
           locate_bytes(w5, m5) + 4 * w5.G * w5.K * w5.C, med, mn, w5.G)
     del Yt, Yt_wm, Yh
     # workload 1: tiny, launch-latency bound

@@ -228,6 +228,30 @@ int approxifer_locate_decode(const approxifer_params* params, int64_t G, int64_t
                              void* cuda_stream);
 
 /*
+ * Scatter / gather variants for the paper's serving architecture (Section 2, "Problem Formulation and System Model":
+ * the coded query i goes to worker i, whose prediction comes back from it): every worker's batch is a buffer of
+ * its own -- on this GPU, or on a peer GPU whose memory is mapped into this process -- instead of a row of one
+ * array.  `Xt_rows` / `Yt_rows` are HOST arrays of W device pointers (read during the call); worker i's buffer holds
+ * its row of group g at element offset g * gstride (gstride >= D or C).  The pointers must be whole elements apart;
+ * 16-byte aligned buffers with D (or C) and the strides multiples of 4 take the 128-bit path.  The encoder computes
+ * every coded row once and stores each to its worker's buffer; the decoder and the locator read each present
+ * worker's row from its buffer (the decoder with its per-column kernel).  Only plain global loads and stores
+ * touch these buffers (no bulk or multicast copies), so peer memory needs nothing but peer access enabled by the
+ * caller.  Formulas, masks, outputs, status bits and return codes as in approxifer_encode / _decode / _locate;
+ * APPROXIFER_E_NULL also if one of the W pointers is NULL or not a whole number of elements from the first.
+ */
+int approxifer_encode_scatter(const approxifer_params* params, int64_t G, int64_t D,
+                              const float* X, int64_t x_gstride, int64_t x_rstride,
+                              float* const* Xt_rows, int64_t xt_gstride, void* cuda_stream);
+int approxifer_decode_gather(const approxifer_params* params, int64_t G, int64_t C,
+                             const float* const* Yt_rows, int64_t yt_gstride, const uint32_t* mask,
+                             float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                             int32_t* n_used, uint32_t* status, void* cuda_stream);
+int approxifer_locate_gather(const approxifer_params* params, int64_t G, int64_t C,
+                             const float* const* Yt_rows, int64_t yt_gstride, const uint32_t* mask,
+                             int32_t* adv, uint32_t* trusted_mask, uint32_t* status, void* cuda_stream);
+
+/*
  * Host-buffer variants of the three operations (same definitions and citations
  * as above).  Payloads, masks and results live in HOST memory, dense
  * ([G][K][D], [G][W][D], [G][W][C], [G][K][C], [G][E], [G]); pinned memory is

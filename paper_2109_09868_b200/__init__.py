@@ -10,6 +10,9 @@ from .binding import (  # noqa: F401
     approxifer_debug_weights,
     approxifer_decode,
     approxifer_decode_bf16,
+    approxifer_decode_gather,
+    approxifer_encode_scatter,
+    approxifer_locate_gather,
     approxifer_encode_bf16,
     approxifer_decode_rational,
     approxifer_encode,

@@ -44,6 +44,9 @@ EXPORTS = (
     "approxifer_locate_host",
     "approxifer_encode_host_static",
     "approxifer_debug_fma_peak",
+    "approxifer_encode_scatter",
+    "approxifer_decode_gather",
+    "approxifer_locate_gather",
     "approxifer_encode_bf16",
     "approxifer_decode_bf16",
 )
@@ -96,6 +99,14 @@ def load() -> ctypes.CDLL:
     lib.approxifer_encode_bf16.restype = c_int
     lib.approxifer_decode_bf16.argtypes = lib.approxifer_decode.argtypes
     lib.approxifer_decode_bf16.restype = c_int
+    lib.approxifer_encode_scatter.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, POINTER(c_void_p), c_int64, c_void_p]
+    lib.approxifer_encode_scatter.restype = c_int
+    lib.approxifer_decode_gather.argtypes = [pp, c_int64, c_int64, POINTER(c_void_p), c_int64, c_void_p, c_void_p, c_int64, c_int64,
+                                             c_void_p, c_void_p, c_void_p]
+    lib.approxifer_decode_gather.restype = c_int
+    lib.approxifer_locate_gather.argtypes = [pp, c_int64, c_int64, POINTER(c_void_p), c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                                             c_void_p]
+    lib.approxifer_locate_gather.restype = c_int
     lib.approxifer_locate.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]
     lib.approxifer_locate.restype = c_int
@@ -298,6 +309,59 @@ def approxifer_locate(params: approxifer_params, Yt: torch.Tensor, mask: torch.T
     if rc != OK:
         raise ApproxiferError(rc, "approxifer_locate")
     return adv, trusted_mask
+
+
+def _row_buffers(rows, W: int, G: int, name: str):
+    """W per-worker CUDA tensors [G][L] (innermost contiguous, same group stride) -> (pointer array, group stride, L)."""
+    if len(rows) != W:
+        raise ValueError("%s must hold one tensor per worker" % name)
+    L, gs = rows[0].shape[1], rows[0].stride(0)
+    for t in rows:
+        if not t.is_cuda or t.dtype != torch.float32 or t.dim() != 2 or t.shape != (G, L) or t.stride(0) != gs or (L > 1 and t.stride(1) != 1):
+            raise ValueError("%s: every worker's batch must be a float32 CUDA tensor [G][L] with the same group stride" % name)
+    return (c_void_p * W)(*[t.data_ptr() for t in rows]), gs, L
+
+
+def approxifer_encode_scatter(params: approxifer_params, X: torch.Tensor, Xt_rows, stream=None) -> None:
+    """X [G][K][D] -> W per-worker batches Xt_rows[i] [G][D] (tensors of their own, possibly in peer memory)."""
+    G, K, D = X.shape
+    xp, xg, xr = _payload(X, params.K, "X")
+    arr, gs, L = _row_buffers(Xt_rows, params.W, G, "Xt_rows")
+    if L != D:
+        raise ValueError("Xt_rows[i] must be [G][D]")
+    rc = load().approxifer_encode_scatter(ctypes.byref(params), G, D, xp, xg, xr, arr, gs, _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_encode_scatter")
+
+
+def approxifer_decode_gather(params: approxifer_params, Yt_rows, mask: torch.Tensor, Yhat: Optional[torch.Tensor] = None,
+                             n_used: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """W per-worker prediction batches Yt_rows[i] [G][C], mask [G] -> Yhat [G][K][C]."""
+    G = Yt_rows[0].shape[0]
+    arr, gs, C = _row_buffers(Yt_rows, params.W, G, "Yt_rows")
+    if Yhat is None:
+        Yhat = torch.empty((G, params.K, C), device=Yt_rows[0].device, dtype=torch.float32)
+    op, og, orr = _payload(Yhat, params.K, "Yhat")
+    rc = load().approxifer_decode_gather(ctypes.byref(params), G, C, arr, gs, _vec(mask, torch.int32, G, "mask"), op, og, orr,
+                                         _vec(n_used, torch.int32, G, "n_used"), _vec(status, torch.int32, G, "status"),
+                                         _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_decode_gather")
+    return Yhat
+
+
+def approxifer_locate_gather(params: approxifer_params, Yt_rows, mask: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None):
+    """W per-worker prediction batches Yt_rows[i] [G][C], mask [G] -> (adv [G][E], trusted_mask [G])."""
+    G = Yt_rows[0].shape[0]
+    arr, gs, C = _row_buffers(Yt_rows, params.W, G, "Yt_rows")
+    E = max(int(params.E), 0)
+    adv = torch.empty((G, E), device=Yt_rows[0].device, dtype=torch.int32)
+    trusted = torch.empty((G,), device=Yt_rows[0].device, dtype=torch.int32)
+    rc = load().approxifer_locate_gather(ctypes.byref(params), G, C, arr, gs, _vec(mask, torch.int32, G, "mask"), adv.data_ptr(),
+                                         trusted.data_ptr(), _vec(status, torch.int32, G, "status"), _stream_ptr(stream))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_locate_gather")
+    return adv, trusted
 
 
 def approxifer_decode_rational(params: approxifer_params, Yt: torch.Tensor, mask: torch.Tensor, Yhat: Optional[torch.Tensor] = None,

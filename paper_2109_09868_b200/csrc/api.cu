@@ -143,6 +143,66 @@ int approxifer_decode_bf16(const approxifer_params* params, int64_t G, int64_t C
   return from_cuda(launch_decode(a, static_cast<cudaStream_t>(cuda_stream)));
 }
 
+namespace {
+// Element offsets of W row pointers from the first one (same address space: device memory of this GPU or of a
+// peer); false if a pointer is missing or not a whole number of elements away.
+bool row_offsets(const float* const* rows, int W, RowOffsets* out) {
+  if (rows == nullptr) return false;
+  for (int i = 0; i < W; ++i) {
+    if (rows[i] == nullptr) return false;
+    const intptr_t diff = reinterpret_cast<intptr_t>(rows[i]) - reinterpret_cast<intptr_t>(rows[0]);
+    if (diff % (intptr_t)sizeof(float) != 0) return false;
+    out->off[i] = (int64_t)(diff / (intptr_t)sizeof(float));
+  }
+  for (int i = W; i < kMaxW; ++i) out->off[i] = 0;
+  out->on = 1;
+  return true;
+}
+}  // namespace
+
+int approxifer_encode_scatter(const approxifer_params* params, int64_t G, int64_t D, const float* X, int64_t x_gstride,
+                              int64_t x_rstride, float* const* Xt_rows, int64_t xt_gstride, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if ((rc = check_layout(G, D, x_rstride))) return rc;
+  if (x_gstride < 0 || xt_gstride < D) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (X == nullptr || Xt_rows == nullptr) return APPROXIFER_E_NULL;
+  EncodeArgs a{X, Xt_rows[0], x_gstride, x_rstride, xt_gstride, D, G, D, params->K, params->W};
+  if (!row_offsets(Xt_rows, params->W, &a.rows)) return APPROXIFER_E_NULL;
+  return from_cuda(launch_encode(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int approxifer_decode_gather(const approxifer_params* params, int64_t G, int64_t C, const float* const* Yt_rows,
+                             int64_t yt_gstride, const uint32_t* mask, float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
+                             int32_t* n_used, uint32_t* status, void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if ((rc = check_layout(G, C, yh_rstride))) return rc;
+  if (G < 0 || C < 1 || yt_gstride < C || yh_gstride < 0) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (Yt_rows == nullptr || Yhat == nullptr || mask == nullptr) return APPROXIFER_E_NULL;
+  DecodeArgs a{Yt_rows[0], mask, Yhat, n_used, status, yt_gstride, C, yh_gstride, yh_rstride, G, C, params->K, params->W, params->flags};
+  if (!row_offsets(Yt_rows, params->W, &a.rows)) return APPROXIFER_E_NULL;
+  return from_cuda(launch_decode(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int approxifer_locate_gather(const approxifer_params* params, int64_t G, int64_t C, const float* const* Yt_rows,
+                             int64_t yt_gstride, const uint32_t* mask, int32_t* adv, uint32_t* trusted_mask, uint32_t* status,
+                             void* cuda_stream) {
+  int rc = check_kw(params);
+  if (rc) return rc;
+  if (params->E < 0) return APPROXIFER_E_RANGE;
+  if (params->E < 1 || 2 * (params->K + params->E) > params->W) return APPROXIFER_E_PARAM;
+  if ((params->flags & APPROXIFER_LOCATE_HOMOGENEOUS) && params->K + params->E > kLocateAltMaxM) return APPROXIFER_E_PARAM;
+  if (G < 0 || C < 1 || C > (int64_t(1) << 31) || yt_gstride < C) return APPROXIFER_E_RANGE;
+  if (G == 0) return APPROXIFER_OK;
+  if (Yt_rows == nullptr || mask == nullptr || adv == nullptr || trusted_mask == nullptr) return APPROXIFER_E_NULL;
+  LocateArgs a{Yt_rows[0], mask, adv, trusted_mask, status, yt_gstride, C, G, C, params->K, params->W, params->E, params->flags};
+  if (!row_offsets(Yt_rows, params->W, &a.rows)) return APPROXIFER_E_NULL;
+  return from_cuda(launch_locate(a, static_cast<cudaStream_t>(cuda_stream)));
+}
+
 int approxifer_debug_decode(const approxifer_params* params, int64_t G, int64_t C, const float* Yt, int64_t yt_gstride,
                             int64_t yt_rstride, const uint32_t* mask, float* Yhat, int64_t yh_gstride, int64_t yh_rstride,
                             int32_t* n_used, uint32_t* status, const approxifer_decode_tuning* tuning, void* cuda_stream) {

@@ -19,6 +19,14 @@ constexpr uint32_t kStTimeout = 16u;
 constexpr uint32_t kFlagSignWorkerIndex = 1u;
 constexpr uint32_t kFlagLocateHomogeneous = 2u;
 
+// Rows of a group that are not a fixed stride apart: off[i] = element offset of worker i's row of group 0 from the
+// base pointer (the rows of one worker for consecutive groups are still `gstride` apart).  Used by the scatter /
+// gather entry points, where every worker's batch is a buffer of its own.
+struct RowOffsets {
+  int64_t off[kMaxW];
+  int32_t on = 0;
+};
+
 struct EncodeArgs {
   const float* X;  // (bfloat16 payloads: really const uint16_t*, see `bf16`)
   float* Xt;
@@ -26,6 +34,7 @@ struct EncodeArgs {
   int64_t G, D;
   int32_t K, W;
   int32_t bf16 = 0;  // payload elements are bfloat16 (2 bytes) instead of fp32; weights and sums stay fp32
+  RowOffsets rows;   // (scatter) where the W coded rows go, instead of o_rs apart
 };
 
 // Test / tuning choices of one decode call (all zero = automatic); see approxifer_debug_decode.
@@ -54,6 +63,7 @@ struct DecodeArgs {
   uint32_t flags;
   DecodeTuning tune = {};
   int32_t bf16 = 0;  // Yt and Yh hold bfloat16 elements (2 bytes); weights and sums stay fp32
+  RowOffsets rows;   // (gather) where the W coded rows are, instead of y_rs apart
 };
 
 struct LocateArgs {
@@ -74,6 +84,7 @@ struct LocateArgs {
   int32_t fuse_decode = 0;
   int32_t* n_used = nullptr;          // decode's optional outputs
   uint32_t* decode_status = nullptr;
+  RowOffsets rows;                    // (gather) where the W coded rows are, instead of y_rs apart
 };
 
 // Each returns a cudaError_t from the launch (cudaSuccess if nothing to do).

@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
       V y[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u)
-        if ((bits >> u) & 1u) y[u] = P::load(in + (i0 + u) * in_rs);
+        if ((bits >> u) & 1u) y[u] = P::load(in + (a.rows.on ? a.rows.off[i0 + u] / Ops::kLanes : (i0 + u) * in_rs));
 #pragma unroll
       for (int u = 0; u < 8; ++u)
         if ((bits >> u) & 1u) {
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const __grid_con
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u)
-        if (i[u] >= 0) y[u] = P::load(in + i[u] * in_rs);
+        if (i[u] >= 0) y[u] = P::load(in + (a.rows.on ? a.rows.off[i[u]] / Ops::kLanes : i[u] * in_rs));
 #pragma unroll
       for (int u = 0; u < 4; ++u)
         if (i[u] >= 0) use_row(i[u], r + u, y[u]);
@@ -228,7 +228,12 @@ __global__ void debug_encode_weights_kernel(int K, int W, const __grid_constant_
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   const DecodeTables& tab = decode_tables(a.K, a.W);
-  const bool by4 = a.C % 4 == 0 && a.y_gs % 4 == 0 && a.y_rs % 4 == 0 && a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  bool by4 = a.C % 4 == 0 && a.y_gs % 4 == 0 && (a.rows.on || a.y_rs % 4 == 0) && a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  if (a.rows.on) {  // gathered rows: the per-column kernel follows the offset table
+    for (int i = 0; i < a.W; ++i) by4 = by4 && a.rows.off[i] % 4 == 0;
+    if (by4 && aligned16(a.Yt) && aligned16(a.Yh)) return dispatch_k<PayloadF32x4>(a, tab, stream);
+    return dispatch_k<PayloadF32>(a, tab, stream);
+  }
   if (a.bf16) {  // bfloat16 payloads: the bulk-copy staged kernel for long rows, else the per-column kernel, four
                  // elements (8 bytes) per thread where it can
     if (decode_staged_eligible(a)) return launch_decode_staged(a, tab, stream);

@@ -52,7 +52,8 @@ struct VecOps<float> {
 // One work item = (group g, column v) with v counting V-wide columns of the
 // payload; items are numbered g*Dv + v and dealt to threads in order, so a
 // warp reads and writes 32 consecutive columns of a row.
-template <int K, typename P, int THREADS>
+// SCATTER: the W coded rows go to per-worker buffers (an offset table) instead of rows a fixed stride apart.
+template <int K, typename P, int THREADS, bool SCATTER = false>
 __global__ void __launch_bounds__(THREADS) encode_kernel(const __grid_constant__ EncodeArgs a,
                                                          const __grid_constant__ EncodeTables tab) {
   using V = typename P::Vec;
@@ -82,7 +83,8 @@ __global__ void __launch_bounds__(THREADS) encode_kernel(const __grid_constant__
     V acc = Ops::mul(wi[0], x[0]);
 #pragma unroll
     for (int j = 1; j < K; ++j) acc = Ops::fma(wi[j], x[j], acc);
-    P::store(out + i * out_rs, acc);
+    if constexpr (SCATTER) P::store(out + a.rows.off[i] / Ops::kLanes, acc);
+    else P::store(out + i * out_rs, acc);
   }
 }
 
@@ -95,6 +97,13 @@ cudaError_t launch_one(const EncodeArgs& a, const EncodeTables& tab, cudaStream_
   // size: each CTA then reads and writes whole contiguous pieces of K and W rows, which HBM serves slightly
   // better (+0.8 % on workload 2) than the 4 KB pieces of 256-thread CTAs.
   // (K <= 16: beyond that 768 threads do not leave a thread enough registers for its K inputs)
+  if (a.rows.on) {
+    const int64_t blocks = (items + kEncodeThreads - 1) / kEncodeThreads;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    encode_kernel<K, V, kEncodeThreads, true><<<(unsigned)blocks, kEncodeThreads, 0, stream>>>(a, tab);
+    count_launch();
+    return cudaGetLastError();
+  }
   if constexpr (P::kLanes == 4 && K <= 16) {  // (16-byte columns of fp32, 8-byte columns of bfloat16)
     if (Dv % kEncodeWideThreads == 0) {
       const int64_t blocks = items / kEncodeWideThreads;
@@ -152,9 +161,11 @@ cudaError_t launch_fma_peak(int iters, int blocks, float* sink, cudaStream_t str
 cudaError_t launch_encode(const EncodeArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   const EncodeTables& tab = encode_tables(a.K, a.W);
-  const bool by4 = a.D % 4 == 0 && a.x_gs % 4 == 0 && a.x_rs % 4 == 0 && a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
+  bool by4 = a.D % 4 == 0 && a.x_gs % 4 == 0 && a.x_rs % 4 == 0 && a.o_gs % 4 == 0 && (a.rows.on || a.o_rs % 4 == 0);
+  if (a.rows.on)
+    for (int i = 0; i < a.W; ++i) by4 = by4 && a.rows.off[i] % 4 == 0;
   if (a.bf16) {  // eight bfloat16 elements are one 16-byte column (K <= 16: a thread keeps 8 K inputs), four an 8-byte one
-    const bool by8 = a.D % 8 == 0 && a.x_gs % 8 == 0 && a.x_rs % 8 == 0 && a.o_gs % 8 == 0 && a.o_rs % 8 == 0;
+    const bool by8 = a.D % 8 == 0 && a.x_gs % 8 == 0 && a.x_rs % 8 == 0 && a.o_gs % 8 == 0 && a.o_rs % 8 == 0 && !a.rows.on;
     if (by8 && a.K <= 16 && aligned16(a.X) && aligned16(a.Xt)) return dispatch_k<PayloadBf16x8>(a, tab, stream);
     if (by4 && aligned8(a.X) && aligned8(a.Xt)) return dispatch_k<PayloadBf16x4>(a, tab, stream);
     return dispatch_k<PayloadBf16>(a, tab, stream);

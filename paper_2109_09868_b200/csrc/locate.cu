@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(kLocateThreads) locate_kernel(const __grid_con
   if (lane < NMAX) {
     const double b = (lane < n) ? tab.beta[my_worker] : 0.0;
     sm.xs[lane] = b;
-    sm.yoff[lane] = (lane < n) ? (long long)my_worker * a.y_rs : 0;
+    sm.yoff[lane] = (lane < n) ? (a.rows.on ? (long long)a.rows.off[my_worker] : (long long)my_worker * a.y_rs) : 0;
     double p = 1.0;
 #pragma unroll
     for (int k = 0; k < M; ++k) {

@@ -204,7 +204,7 @@ __device__ __forceinline__ void rows_setup_group(GroupSmem<NMAX, M>& sm, double 
   if (lane < NMAX) {
     const double b = (lane < n) ? tab.beta[my_worker] : 0.0;
     sm.xs[lane] = b;
-    sm.yoff[lane] = (lane < n) ? (long long)my_worker * a.y_rs : 0;
+    sm.yoff[lane] = (lane < n) ? (a.rows.on ? (long long)a.rows.off[my_worker] : (long long)my_worker * a.y_rs) : 0;
     double p = 1.0;
 #pragma unroll
     for (int k = 0; k < SM::MP; ++k) {
