@@ -47,11 +47,11 @@ HEADLINE_CFG = 3
 HEADLINE_NAME = "configs[2]: K=12 W=20 D=150528 (3x224x224) C=1000, Bernoulli(0.3) stragglers capped at 8"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# DRAM traffic (ncu dram__bytes_read.sum + dram__bytes_write.sum) of encode_kernel<12, float4, 768> per group of
+# DRAM traffic (ncu dram__bytes_read.sum + dram__bytes_write.sum) of encode_kernel<12, PayloadF32x4, 768> per group of
 # the headline workload, from a capture of a reduced launch (profiles/encode_kernel_K12_W20_D150528.md); traffic is
 # proportional to the number of groups (every row is touched once).  Set to None when the kernel changes, until
 # the counters have been taken again.
-ENCODE_TRAFFIC_PER_GROUP = (1387302912 + 2254066944) / 192
+ENCODE_TRAFFIC_PER_GROUP = (1387421696 + 2254734336) / 192
 ENCODE_TRAFFIC_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of a 192-group launch (3.7 GB) of the unchanged kernel, "
                          "per group x groups; the written part misses the ~58 MB of dirty lines still in L2 at kernel end")
 E2E_GROUPS = 256
