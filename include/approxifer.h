@@ -236,7 +236,7 @@ int approxifer_locate_decode(const approxifer_params* params, int64_t G, int64_t
  * 16-byte aligned buffers with D (or C) and the strides multiples of 4 take the 128-bit path.  The encoder computes
  * every coded row once and stores each to its worker's buffer; the decoder and the locator read each present
  * worker's row from its buffer (the decoder with its per-column kernel).  Only plain global loads and stores
- * touch these buffers (no bulk or multicast copies), so peer memory needs nothing but peer access enabled by the
+ * touch these buffers (no bulk asynchronous copies), so peer memory needs nothing but peer access enabled by the
  * caller.  Formulas, masks, outputs, status bits and return codes as in approxifer_encode / _decode / _locate;
  * APPROXIFER_E_NULL also if one of the W pointers is NULL or not a whole number of elements from the first.
  */
