@@ -343,8 +343,10 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
  *   cols         ... 16, 32 (split 2 only), 64, 128 or 256 16-byte columns per work item (256 needs split 1 or 2
  *                and a ring that fits in shared memory, else 128 is used)
  *   split        ... 1 (K <= 16, 256 columns), 2 or 4 thread groups sharing the K queries of a column
- *   For the packed-groups kernel (dense buffers, even C <= 62) `stages` = 2..4 sets each warp's ring depth,
- *   `ctas_per_sm` bounds the warps per CTA and `cols` (any positive value) the groups per work item.
+ *   For the packed-groups kernel (dense buffers, even C <= 62) `ctas_per_sm` bounds the warps per CTA, `cols`
+ *   (any positive value) the groups per work item, and `split` = 1 / 2 switches off / on the rotated word order
+ *   that keeps a warp's lanes in different shared-memory banks (0: where it measured faster); `stages` is ignored
+ *   (each warp's ring has two slots).
  * APPROXIFER_E_PARAM for any other value.
  *
  * Exercising the bounded waits.  The two decoders that stage predictions with asynchronous copies (bulk-copy

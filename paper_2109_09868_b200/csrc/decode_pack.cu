@@ -9,8 +9,8 @@
 //  * Every WARP is a pipeline of its own.  A warp's work item is a block of GW consecutive groups (a few KB,
 //    one contiguous range: rows this short are shorter than a DRAM burst, so the absent workers' rows come
 //    along and are simply never used).  Lane 0 brings items into the warp's private shared-memory ring with
-//    bulk asynchronous copies, S-1 items ahead of the one being reduced, completion counted on one mbarrier
-//    per slot; a slot is refilled by the warp that has just finished reading it, so there are no "empty"
+//    bulk asynchronous copies, one item ahead of the one being reduced (the ring has two slots: deeper rings
+//    measured slower, and cost registers), completion counted on one mbarrier per slot; a slot is refilled by the warp that has just finished reading it, so there are no "empty"
 //    barriers, no producer warp and no CTA-wide barrier in the main loop.  With a dozen such warps per SM
 //    there are always tens of KB of loads in flight and always some warp with arithmetic to do.
 //  * Lane = (group of the item, tile of two queries, word lane).  A thread forms two queries for NW words
@@ -23,8 +23,18 @@
 //    K rows never take more room than W) and streamed out by the whole warp with 128-bit stores, again one
 //    contiguous range.  (A bulk copy out of shared memory frees its source only after
 //    several microseconds; waiting for that dominated every variant that used one.)
+//  * The masks of an item come with it: a second bulk copy on the same mbarrier brings the 16-byte columns of
+//    the mask array that hold them (an ordinary load per item cost a tenth of the run time).
+//  * Shared memory, not DRAM, bounds this kernel (its load/store pipe is 60-80 % busy), and an item's groups are
+//    as far apart in shared memory as in DRAM, so groups can start in the same banks.  Where they do, some
+//    groups take the words of their rows in an order rotated by one (register slot u holds word u + 1), which
+//    puts the lanes that execute the same load or store into different banks; the host picks the groups with a
+//    model of the bank rules (see choose_rotation).
 //
 // Every wait is bounded.  Every bulk copy targets, or reads, the issuing CTA's own shared memory.
+#include <mutex>
+#include <vector>
+
 #include "common.cuh"
 
 namespace approxifer {
@@ -35,9 +45,10 @@ namespace {
 
 constexpr int kPackMaxWarps = 24;  // 768 threads: 80 registers each
 __host__ __device__ constexpr int pack_max_warps(int) { return kPackMaxWarps; }
-constexpr int kPackMaxStages = 4;
+constexpr int kPackStages = 2;  // ring slots per warp
 constexpr int kPackMaxNW = 5;  // words (float2) per thread and row
 constexpr int kPackMaxC = 62;
+constexpr int kPackMaskBytes = 160;  // up to 32 masks, widened to whole 16-byte columns of the mask array
 constexpr uint32_t kPackWaitLimit = 1u << 22;
 constexpr unsigned kFullMask = 0xffffffffu;
 
@@ -99,43 +110,53 @@ struct PackPlan {
   int32_t gw;         // groups per warp item
   int32_t nch;        // lanes sharing the words of one (group, query tile)
   int32_t jt;         // query tiles per group = ceil(K / 2)
-  int32_t stages;     // ring depth per warp
   int32_t warps;      // warps per CTA
-  int32_t in_bytes;   // one ring slot (gw * W * C floats, padded to 128 B)
+  int32_t in_bytes;   // one ring slot: gw * W * C floats padded to 128 B, then the item's masks (kPackMaskBytes)
+  int32_t mask_off;   // where a slot's masks start
   int32_t table_bytes;
+  // sizes the kernel would otherwise keep in registers (as kernel parameters they are read where they are used)
+  uint32_t row_bytes;      // C floats
+  uint32_t group_bytes;    // W rows
+  uint32_t result_bytes;   // K rows
+  uint32_t wrow_bytes;     // one worker's row of the weight table: KP entries of 8 bytes
+  uint32_t sign_bytes;     // between the two signs of the weight table (padded: the two copies of a row sit in
+                           // different halves of the banks, since the lanes of a warp read both at once)
+  uint32_t coin_off;       // where coin[32] starts
+  uint32_t rot_groups;     // bit s: the lanes of the item's group s keep their row's words rotated by one
+  uint32_t wait_limit;     // probes of a wait before it gives up
+  int32_t probe;           // (test hook) non-blocking probes
   int64_t n_items;
 };
 
 __device__ __forceinline__ float p_lo(uint64_t v) { return __uint_as_float((uint32_t)v); }
 __device__ __forceinline__ float p_hi(uint64_t v) { return __uint_as_float((uint32_t)(v >> 32)); }
 
-// Shared memory: wtab[2][W][KP] (8 bytes each) | coin[32] | per warp: full[S] mbarriers (64 B) | S ring slots.
+// Shared memory: wtab[2][W][KP] (8 bytes each) | coin[32] | per warp: full[2] mbarriers (64 B) | 2 ring slots.
 // wtab[sg][i][j] = (w, w) with w = (-1)^sg / (alpha_j - beta_i): the signed weight, already duplicated for the
 // packed multiply-add (the sign flip is exact, so (s rg) y rounds like rg (s y)).
 // SIMPLE: one lane owns all the words of its rows (nch == 1, NW == C/2), so every offset is a compile-time constant.
-template <int NW, bool SIMPLE>
+template <int NW, bool SIMPLE, bool ROT>
 __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     decode_pack_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ DecodeTables tab,
                        const __grid_constant__ PackPlan plan) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int W = a.W, K = a.K, C = (int)a.C, S = plan.stages, GW = plan.gw;
+  const int W = a.W, K = a.K, C = (int)a.C, GW = plan.gw;
+  constexpr int S = kPackStages;
   const int KP = (K + 1) & ~1;
-  uint64_t* wtab = reinterpret_cast<uint64_t*>(smem_raw);           // [2][W][KP], 0 beyond K
-  int* coins = reinterpret_cast<int*>(smem_raw + 2 * W * KP * 8);  // [32]
+  uint64_t* wtab = reinterpret_cast<uint64_t*>(smem_raw);    // [2][W][KP], 0 beyond K
+  int* coins = reinterpret_cast<int*>(smem_raw + plan.coin_off);  // [32]
   const uint32_t per_warp = 64u + (uint32_t)S * (uint32_t)plan.in_bytes;
   unsigned char* mine = smem_raw + plan.table_bytes + (size_t)warp * per_warp;
   uint64_t* full = reinterpret_cast<uint64_t*>(mine);
   unsigned char* slots = mine + 64;
   const uint32_t wb = worker_bits(W);
-  const uint32_t group_bytes = (uint32_t)(W * C * 4);
-  const uint32_t row_bytes = (uint32_t)(C * 4);
 
   for (int idx = tid; idx < 2 * W * KP; idx += blockDim.x) {
     const int sg = idx / (W * KP), rem = idx - sg * (W * KP);
     const int i = rem / KP, j = rem - i * KP;
     const float w = (j < K) ? tab.rg[i * K + j] : 0.f;
-    wtab[idx] = p_dup(sg ? -w : w);
+    wtab[(sg ? plan.sign_bytes / 8u : 0u) + (uint32_t)rem] = p_dup(sg ? -w : w);
   }
   if (tid < 32) coins[tid] = (tab.any_coin && tid < K) ? (int)tab.coin[tid] : -1;
   if (lane == 0) {
@@ -156,75 +177,81 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
   const int Cw = C >> 1;
   const bool exact = SIMPLE || NW * nch == Cw;  // no lane has a word beyond the end of the row
   const bool literal = (a.flags & kFlagSignWorkerIndex) != 0;
-  const uint32_t y_off = (uint32_t)s * group_bytes + (uint32_t)ch * 8u;
+  const uint32_t y_off = (uint32_t)s * plan.group_bytes + (uint32_t)ch * 8u;
+  const uint32_t o_off = (uint32_t)(s * K + j0) * plan.row_bytes + (uint32_t)ch * 8u;
   const uint32_t u_step = (uint32_t)nch * 8u;
+  // Where register slot u's word sits in a row.  With one lane per row (SIMPLE) the groups whose rows start in the
+  // same banks as an earlier group's take their words in rotated order (slot u holds word (u + 1) mod NW), so
+  // that the lanes of a warp, which all load slot u at once, touch different banks.
+  const bool rot = ROT && ((plan.rot_groups >> s) & 1u);
+  const uint32_t rot8 = rot ? 8u : 0u, last_off = rot ? 0u : (uint32_t)(NW - 1) * 8u;
+  auto woff = [&](int u) -> uint32_t {
+    if constexpr (SIMPLE && ROT) return u < NW - 1 ? (uint32_t)u * 8u + rot8 : last_off;
+    else if constexpr (SIMPLE) return (uint32_t)u * 8u;
+    else return (uint32_t)u * u_step;
+  };
   const int c0 = (j0 < K) ? coins[j0] : -1, c1 = (j0 + 1 < K) ? coins[j0 + 1] : -1;
-  const uint32_t sign_step = (uint32_t)(W * KP) * 8u;  // bytes between the two signs of the table
   const unsigned char* wrow0 = reinterpret_cast<const unsigned char*>(wtab) + (uint32_t)j0 * 8u;
 
   // lane 0: start the copy of the item whose first group is g0 into ring slot `slot`.  A ragged last item may end
   // on an 8-byte boundary: the copy takes the whole 16-byte columns and the last two floats go by hand.
   auto issue = [&](int64_t g0, int slot) {
     const int ng = (int)min((int64_t)GW, a.G - g0);
-    const uint32_t bytes = (uint32_t)ng * group_bytes, bytes16 = bytes & ~15u;
-    const unsigned char* src = reinterpret_cast<const unsigned char*>(a.Yt + g0 * (int64_t)(W * C));
+    const uint32_t bytes = (uint32_t)ng * plan.group_bytes, bytes16 = bytes & ~15u;
+    const unsigned char* src = reinterpret_cast<const unsigned char*>(a.Yt) + g0 * (int64_t)plan.group_bytes;
     unsigned char* dst = slots + (size_t)slot * plan.in_bytes;
     const uint32_t bar = p_smem_u32(full + slot);
     // (test hook: the item that holds one chosen group is never fetched, so the wait for it runs out)
     if (a.tune.withhold_group >= g0 && a.tune.withhold_group < g0 + ng) return;
     if (bytes16 != bytes) *reinterpret_cast<float2*>(dst + bytes16) = *reinterpret_cast<const float2*>(src + bytes16);
-    p_arrive_expect_tx(bar, bytes16);  // (release: the two floats above are visible to whoever sees the phase complete)
+    // the item's masks travel the same way: the whole 16-byte columns of the mask array that hold them (group g's
+    // mask lands at word (g0 & 3) + g - g0 of the slot's mask area); by hand where those would end beyond the array
+    const int64_t m0 = g0 & ~int64_t(3), m1 = (g0 + ng + 3) & ~int64_t(3);
+    uint32_t mask_bytes = 0;
+    if (m1 <= a.G) mask_bytes = (uint32_t)(m1 - m0) * 4u;
+    else
+      for (int q = 0; q < ng; ++q) reinterpret_cast<uint32_t*>(dst + plan.mask_off)[(int)(g0 & 3) + q] = a.mask[g0 + q];
+    // (release: what was written by hand above is visible to whoever sees the phase complete)
+    p_arrive_expect_tx(bar, bytes16 + mask_bytes);
     if (bytes16) p_bulk_g2s(p_smem_u32(dst), src, bytes16, bar);
+    if (mask_bytes) p_bulk_g2s(p_smem_u32(dst + plan.mask_off), a.mask + m0, mask_bytes, bar);
   };
-  // this lane's group's mask in the item whose first group is g0 (0 beyond the end)
-  auto fetch_mask = [&](int64_t g0) -> uint32_t {
-    const int64_t g = g0 + s;
-    return (s < GW && g < a.G) ? (a.mask[g] & wb) : 0u;
-  };
+  const bool probe = plan.probe != 0;  // (test hook: a short limit, counted in non-blocking probes)
+  // prologue: one item in flight
+  const int64_t g_stride = stride * GW;
+  int left = (int)my_items;  // items this warp has still to reduce (the launch keeps this below 2^31)
+  int64_t g0 = first * GW;   // first group of the item being reduced
+  if (lane == 0 && left > 0) issue(g0, 0);
 
-  const bool probe = a.tune.wait_limit != 0;  // (test hook: a short limit, counted in non-blocking probes)
-  const uint32_t wait_limit = probe ? a.tune.wait_limit : kPackWaitLimit;
-  // prologue: S-1 items in flight, their masks in registers (mq0 belongs to the item about to be reduced)
-  const int64_t g_first = first * GW, g_stride = stride * GW;
-  const int64_t g_end = g_first + my_items * g_stride;  // first group of the item after this warp's last
-  uint32_t mq0 = 0u, mq1 = 0u, mq2 = 0u;
-  if (S > 1 && 0 < my_items) mq0 = fetch_mask(g_first);
-  if (S > 2 && 1 < my_items) mq1 = fetch_mask(g_first + g_stride);
-  if (S > 3 && 2 < my_items) mq2 = fetch_mask(g_first + 2 * g_stride);
-  if (lane == 0)
-    for (int d = 0; d < S - 1 && d < my_items; ++d) issue(g_first + d * g_stride, d);
-
-  int64_t g0 = g_first;                             // first group of the item being reduced
-  int64_t g_ahead = g_first + (S - 1) * g_stride;   // ... of the item started in the same iteration
-  int slot = 0, slot_ahead = S - 1;                 // their ring slots
+  int slot = 0;  // ring slot of the item being reduced; the item started in the same iteration goes to the other
   uint32_t parity = 0;
-  int64_t failed_g0 = -1;
-  for (; g0 < g_end; g0 += g_stride, g_ahead += g_stride) {
+  bool failed = false;
+  for (; left > 0; --left, g0 += g_stride) {
     const int ng = (int)min((int64_t)GW, a.G - g0);
     // the slot that the previous item occupied is free (its results were copied out of it before the __syncwarp
-    // that ended the previous iteration): refill it with the item S-1 ahead, and fetch that item's mask
-    uint32_t m_new = 0u;
-    if (g_ahead < g_end) {
-      m_new = fetch_mask(g_ahead);
-      if (lane == 0) issue(g_ahead, slot_ahead);
-    }
+    // that ended the previous iteration): refill it with the next item
+    if (lane == 0 && left > 1) issue(g0 + g_stride, slot ^ 1);
     // wait for this item's bytes (bounded)
     {
       const uint32_t addr = p_smem_u32(full + slot);
       bool ok = false;
-      for (uint32_t it = 0; it < wait_limit && !ok; ++it) ok = probe ? p_test_wait(addr, parity) : p_try_wait(addr, parity);
+      for (uint32_t it = 0; it < plan.wait_limit && !ok; ++it) ok = probe ? p_test_wait(addr, parity) : p_try_wait(addr, parity);
       if (!__all_sync(kFullMask, ok)) {
         if (lane == 0) atomicAdd(&g_pack_wait_timeouts, 1u);
-        failed_g0 = g0;
+        failed = true;
         // this warp's items from here on are not written: say so in their groups' status words
-        if (a.status != nullptr)
-          for (int64_t q = g0; q < g_end; q += g_stride)
+        if (a.status != nullptr) {
+          int64_t q = g0;
+          for (int c = left; c > 0; --c, q += g_stride)
             if (s < GW && q + s < a.G) a.status[q + s] = kStTimeout;
+        }
         break;
       }
     }
-    const uint32_t mask = mq0;
-    const unsigned char* yg = slots + (size_t)slot * plan.in_bytes + y_off;
+    const unsigned char* slot_base = slots + (size_t)slot * plan.in_bytes;
+    const uint32_t mask =
+        (s < ng) ? (reinterpret_cast<const uint32_t*>(slot_base + plan.mask_off)[(int)(g0 & 3) + s] & wb) : 0u;
+    const unsigned char* yg = slot_base + y_off;
     uint64_t acc0[NW], acc1[NW];  // numerators of this lane's two queries, a pair of classes per word
     float inv0 = 0.f, inv1 = 0.f;
     bool pin0 = false, pin1 = false;
@@ -237,17 +264,16 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
       const unsigned char* yr = yg;
       const unsigned char* wr = wrow0;
 #pragma unroll 2
-      for (int i = 0; i < W; ++i, yr += row_bytes, wr += KP * 8) {
+      for (int i = 0; i < W; ++i, yr += plan.row_bytes, wr += plan.wrow_bytes) {
         uint64_t y[NW];
 #pragma unroll
         for (int u = 0; u < NW; ++u) {  // (an absent worker's row may be loaded; it is only used under `present`)
-          if constexpr (SIMPLE) y[u] = reinterpret_cast<const uint64_t*>(yr)[u];
-          else y[u] = (exact || u * nch + ch < Cw) ? *reinterpret_cast<const uint64_t*>(yr + u * u_step) : 0ull;
+          y[u] = (exact || u * nch + ch < Cw) ? *reinterpret_cast<const uint64_t*>(yr + woff(u)) : 0ull;
         }
         if ((mask >> i) & 1u) {
           // the signed, duplicated weights of this lane's two queries
           const uint32_t odd = (literal ? (uint32_t)i : r) & 1u;
-          const ulonglong2 w2 = *reinterpret_cast<const ulonglong2*>(wr + odd * sign_step);
+          const ulonglong2 w2 = *reinterpret_cast<const ulonglong2*>(wr + odd * plan.sign_bytes);
           den0 = __fadd_rn(den0, p_lo(w2.x));
           den1 = __fadd_rn(den1, p_lo(w2.y));
 #pragma unroll
@@ -266,8 +292,8 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
 #pragma unroll
         for (int u = 0; u < NW; ++u) {
           if (exact || u * nch + ch < Cw) {
-            if (pin0) acc0[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c0 * row_bytes + u * u_step);
-            if (pin1) acc1[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c1 * row_bytes + u * u_step);
+            if (pin0) acc0[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c0 * plan.row_bytes + woff(u));
+            if (pin1) acc1[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c1 * plan.row_bytes + woff(u));
           }
         }
       }
@@ -275,15 +301,15 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     __syncwarp();  // every lane has finished reading the slot: the results take its place
     unsigned char* ob = slots + (size_t)slot * plan.in_bytes;
     if (s < ng) {
-      unsigned char* orow = ob + (size_t)(s * K + j0) * row_bytes + (size_t)ch * 8u;
+      unsigned char* orow = ob + o_off;
 #pragma unroll
       for (int u = 0; u < NW; ++u) {
         if (exact || u * nch + ch < Cw) {
           float2 v0 = pin0 ? make_float2(p_lo(acc0[u]), p_hi(acc0[u])) : make_float2(p_lo(acc0[u]) * inv0, p_hi(acc0[u]) * inv0);
           float2 v1 = pin1 ? make_float2(p_lo(acc1[u]), p_hi(acc1[u])) : make_float2(p_lo(acc1[u]) * inv1, p_hi(acc1[u]) * inv1);
           if (n == 0) v0 = v1 = make_float2(0.f, 0.f);
-          if (j0 < K) *reinterpret_cast<float2*>(orow + u * u_step) = v0;
-          if (j0 + 1 < K) *reinterpret_cast<float2*>(orow + row_bytes + u * u_step) = v1;
+          if (j0 < K) *reinterpret_cast<float2*>(orow + woff(u)) = v0;
+          if (j0 + 1 < K) *reinterpret_cast<float2*>(orow + plan.row_bytes + woff(u)) = v1;
         }
       }
       if (jt == 0 && ch == 0) {
@@ -295,43 +321,34 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     {
       // the item's results are one contiguous range: the warp streams it out in whole 16-byte columns (a ragged
       // last item may end on an 8-byte boundary)
-      const uint32_t bytes = (uint32_t)ng * (uint32_t)(K * C * 4), n16 = bytes >> 4;
-      unsigned char* dst = reinterpret_cast<unsigned char*>(a.Yh + g0 * (int64_t)(K * C));
+      const uint32_t bytes = (uint32_t)ng * plan.result_bytes, n16 = bytes >> 4;
+      unsigned char* dst = reinterpret_cast<unsigned char*>(a.Yh) + g0 * (int64_t)plan.result_bytes;
       for (uint32_t q = lane; q < n16; q += 32)
         st_stream(reinterpret_cast<float4*>(dst) + q, reinterpret_cast<const float4*>(ob)[q]);
       if (lane == 0 && (bytes & 15u))
         __stcs(reinterpret_cast<float2*>(dst + (n16 << 4)), *reinterpret_cast<const float2*>(ob + (n16 << 4)));
     }
     __syncwarp();  // the slot may be refilled
-    // masks move up the queue; the newly fetched one joins at position S-2
-    mq0 = mq1, mq1 = mq2;
-    if (S == 2) mq0 = m_new;
-    else if (S == 3) mq1 = m_new;
-    else mq2 = m_new;
-    slot_ahead = slot;
-    if (++slot == S) {
-      slot = 0;
-      parity ^= 1u;
-    }
+    parity ^= (uint32_t)slot;  // (a slot's phase flips every second item)
+    slot ^= 1;
   }
-  if (lane == 0 && failed_g0 >= 0) {
-    // the copies of the failed item and of the S-1 after it have been started: they must land before the CTA's
+  if (lane == 0 && failed) {
+    // the copies of the failed item and of the one after it have been started: they must land before the CTA's
     // shared memory is given up (bounded)
-    for (int d = 0; d < S && failed_g0 + d * g_stride < g_end; ++d) {
+    for (int d = 0; d < S && d < left; ++d) {
       const uint32_t addr = p_smem_u32(full + slot);
-      for (uint32_t it = 0; it < wait_limit; ++it)
+      for (uint32_t it = 0; it < plan.wait_limit; ++it)
         if (probe ? p_test_wait(addr, parity) : p_try_wait(addr, parity)) break;
-      if (++slot == S) {
-        slot = 0;
-        parity ^= 1u;
-      }
+      parity ^= (uint32_t)slot;
+      slot ^= 1;
     }
   }
 }
 
 struct PackChoice {
-  int nw = 0, nch = 0, jt = 0, gw = 0, stages = 0, warps = 0;
-  int in_bytes = 0, table_bytes = 0, smem = 0;
+  int nw = 0, nch = 0, jt = 0, gw = 0, warps = 0;
+  uint32_t rot_groups = 0;
+  int in_bytes = 0, mask_off = 0, table_bytes = 0, smem = 0;
 };
 
 // How the words of a row are dealt to lanes: NW <= 5 words per lane (more would need more registers than 24 warps
@@ -352,6 +369,121 @@ void choose_words(int Cw, int* nw, int* nch) {
   *nch = (Cw + best_nw - 1) / best_nw;
 }
 
+// Shared-memory cost of an item, in passes of the 32 banks ("wavefronts"), for a given set of rotated groups.
+// The rules are measured ones (64-bit accesses, cycles per instruction with the memory pipe saturated):
+//   loads:  the whole warp at once; lanes reading the same word share it; the cost is the largest number of
+//           different words that fall into one bank;
+//   stores: one half-warp after the other, each costing the largest number of different words in one bank.
+// A row's words are 8-byte aligned, so banks are counted in pairs.  Counted: the W x NW loads of the worker loop
+// (every lane of group s reads word slot u of its row: bytes s * group_bytes + off(u)) and the 2 x NW stores of
+// the results (lane (s, jt): bytes s * result_bytes + jt * 2 * row_bytes + off(u); the second query's row is a
+// uniform shift).  What the rotation cannot change (weights, copy-out) is left out.
+// Returned: passes * 4096 + the number of words beyond the first in every bank (a tie-break that lets a search
+// move across sets with the same number of passes).  A pass of a store counts twice: the stores sit in the
+// dependent tail of an item, between two warp barriers, and measured about that much dearer than the loads of
+// the pipelined worker loop.
+int64_t rotation_cost(int K, int W, int C, int gw, int jt, uint32_t rot_groups, int* passes = nullptr) {
+  const int NW = C / 2;
+  const uint32_t row_bytes = (uint32_t)C * 4u, group_bytes = (uint32_t)W * row_bytes, result_bytes = (uint32_t)K * row_bytes;
+  int loads = 0, stores = 0, excess_loads = 0, excess_stores = 0;
+  for (int u = 0; u < NW; ++u) {
+    uint32_t seen[16][32];  // the different words met so far in each bank pair
+    int n_seen[16];
+    auto reset = [&]() {
+      for (int b = 0; b < 16; ++b) n_seen[b] = 0;
+    };
+    auto touch = [&](uint32_t byte) {
+      const uint32_t word = byte / 8u, b = word % 16u;
+      for (int q = 0; q < n_seen[b]; ++q)
+        if (seen[b][q] == word) return;
+      seen[b][n_seen[b]++] = word;
+    };
+    auto worst = [&]() {
+      int m = 0;
+      for (int b = 0; b < 16; ++b) m = n_seen[b] > m ? n_seen[b] : m;
+      return m;
+    };
+    auto excess = [&]() {
+      int e = 0;
+      for (int b = 0; b < 16; ++b) e += n_seen[b] > 1 ? n_seen[b] - 1 : 0;
+      return e;
+    };
+    auto off = [&](int s) -> uint32_t {
+      const bool rot = (rot_groups >> s) & 1u;
+      return (uint32_t)((u + (rot ? 1 : 0)) % NW) * 8u;
+    };
+    reset();
+    for (int s = 0; s < gw; ++s) touch((uint32_t)s * group_bytes + off(s));
+    loads += worst();
+    excess_loads += excess();
+    for (int half = 0; half < 2; ++half) {
+      reset();
+      for (int lane = half * 16; lane < half * 16 + 16 && lane < gw * jt; ++lane) {
+        const int s = lane / jt, t = lane - s * jt;
+        touch((uint32_t)s * result_bytes + (uint32_t)t * 2u * row_bytes + off(s));
+      }
+      stores += worst();
+      excess_stores += excess();
+    }
+  }
+  if (passes != nullptr) *passes = W * loads + 2 * stores;
+  return (int64_t)(W * loads + 4 * stores) * 4096 + W * excess_loads + 4 * excess_stores;
+}
+
+// Which groups of an item keep the words of their rows rotated by one (kernels with one lane per row): the best of
+// the sets "groups whose index has odd parity under a bit mask", improved by a few rounds of
+// flip-one-group-if-it-helps.  Whether it is used follows what was measured on 18 shapes (K = 2 .. 16,
+// C = 6, 8, 10; 2-3 GB each): with three or more lanes per group (K >= 5) every set the model prefers gained
+// (6-55 %); with one or two lanes per group (K <= 4) it gained (28 %) only where shared memory is what bounds the
+// kernel -- more than one pass per 25 bytes moved -- and cost 5-10 % elsewhere (those shapes already run at the
+// DRAM rate, and the rotated code has a few more instructions); rows of fewer than 8 classes lost either way.
+// The answer depends on the shape alone and is remembered per shape.  mode (tuning): 1 never, 2 whenever the
+// model prefers a set.
+uint32_t choose_rotation(int K, int W, int C, int gw, int jt, int mode) {
+  if (mode == 1 || gw < 2) return 0u;
+  struct Entry {
+    int K, W, C, gw, mode;
+    uint32_t rot;
+  };
+  static std::mutex mu;
+  static std::vector<Entry> memo;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (const Entry& e : memo)
+      if (e.K == K && e.W == W && e.C == C && e.gw == gw && e.mode == mode) return e.rot;
+  }
+  int plain_passes = 0;
+  const int64_t plain = rotation_cost(K, W, C, gw, jt, 0u, &plain_passes);
+  uint32_t best = 0u;
+  int64_t best_cost = plain;
+  for (uint32_t m = 1; m < 32; ++m) {
+    uint32_t cand = 0u;
+    for (int s = 0; s < gw; ++s)
+      if (__builtin_popcount((uint32_t)s & m) & 1) cand |= 1u << s;
+    const int64_t c = rotation_cost(K, W, C, gw, jt, cand);
+    if (c < best_cost) best = cand, best_cost = c;
+  }
+  for (int round = 0; round < 3; ++round) {
+    bool changed = false;
+    for (int s = 0; s < gw; ++s) {
+      const uint32_t cand = best ^ (1u << s);
+      const int64_t c = rotation_cost(K, W, C, gw, jt, cand);
+      if (c < best_cost) best = cand, best_cost = c, changed = true;
+    }
+    if (!changed) break;
+  }
+  // all passes of an item: the counted ones, the weights (about 1.5 per worker) and the copy-out (a load and a
+  // store of every 128 result bytes)
+  const int64_t result_bytes = (int64_t)gw * K * C * 4, moved = (int64_t)gw * W * C * 4 + result_bytes;
+  const int64_t all_passes = plain_passes + (3 * W) / 2 + 2 * (result_bytes / 128);
+  const bool bound_by_shared = all_passes * 25 >= moved;
+  const bool use = best_cost < plain && (mode == 2 || (C >= 8 && (jt >= 3 || bound_by_shared)));
+  const uint32_t rot = use ? best : 0u;
+  std::lock_guard<std::mutex> lock(mu);
+  if (memo.size() < 256) memo.push_back(Entry{K, W, C, gw, mode, rot});
+  return rot;
+}
+
 bool plan_pack(const DecodeArgs& a, int smem_per_sm, PackChoice* out) {
   PackChoice p;
   const int K = a.K, W = a.W, C = (int)a.C;
@@ -368,41 +500,52 @@ bool plan_pack(const DecodeArgs& a, int smem_per_sm, PackChoice* out) {
   if (gw < 1) return false;
   p.gw = gw;
   if (K > W) return false;  // (the results of an item are staged in the slot of its predictions)
-  p.in_bytes = (gw * W * C * 4 + 127) & ~127;
+  if ((a.G + gw - 1) / gw > (int64_t)INT32_MAX) return false;  // (a warp counts its items in 32 bits)
+  p.mask_off = (gw * W * C * 4 + 127) & ~127;
+  p.in_bytes = p.mask_off + kPackMaskBytes;
   const int KP = (K + 1) & ~1;
-  p.table_bytes = (2 * W * KP * 8 + 128 + 127) & ~127;
+  p.table_bytes = (2 * W * KP * 8 + 128 + 128 + 127) & ~127;  // two copies, up to 120 B between them, coin[32]
   const int budget = smem_per_sm - 1024 - p.table_bytes;
   // Two slots per warp: one item in flight while one is reduced.  What hides the latency of the loads is the
   // number of warps (each with an item in flight), not the depth of a warp's ring: measured, 22 warps with two
   // slots beat 16 with three and 12 with four.
-  int stages = 2;
-  if (a.tune.stages >= 2 && a.tune.stages <= kPackMaxStages) stages = a.tune.stages;
-  const int per_warp = 64 + stages * p.in_bytes;
+  const int per_warp = 64 + kPackStages * p.in_bytes;
   int warps = budget / per_warp;
   if (warps > pack_max_warps(p.nw)) warps = pack_max_warps(p.nw);
   if (a.tune.ctas_per_sm > 0 && a.tune.ctas_per_sm < warps) warps = a.tune.ctas_per_sm;  // (tuning: warps per CTA)
   if (warps < 4) return false;
-  p.stages = stages;
   p.warps = warps;
+  if (p.nch == 1 && p.nw * 2 == C) p.rot_groups = choose_rotation(K, W, C, gw, p.jt, a.tune.split);
   p.smem = p.table_bytes + warps * per_warp;
   *out = p;
   return true;
 }
 
-template <int NW, bool SIMPLE>
+template <int NW, bool SIMPLE, bool ROT>
 cudaError_t launch_pack(const DecodeArgs& a, const DecodeTables& tab, const PackChoice& c, const DeviceInfo& di,
                         cudaStream_t stream) {
   PackPlan plan;
-  plan.gw = c.gw, plan.nch = c.nch, plan.jt = c.jt, plan.stages = c.stages, plan.warps = c.warps;
-  plan.in_bytes = c.in_bytes, plan.table_bytes = c.table_bytes;
+  plan.gw = c.gw, plan.nch = c.nch, plan.jt = c.jt, plan.warps = c.warps;
+  plan.in_bytes = c.in_bytes, plan.mask_off = c.mask_off, plan.table_bytes = c.table_bytes;
   plan.n_items = (a.G + c.gw - 1) / c.gw;
+  const int KP = (a.K + 1) & ~1;
+  plan.row_bytes = (uint32_t)a.C * 4u;
+  plan.group_bytes = (uint32_t)a.W * plan.row_bytes;
+  plan.result_bytes = (uint32_t)a.K * plan.row_bytes;
+  plan.wrow_bytes = (uint32_t)KP * 8u;
+  plan.sign_bytes = (uint32_t)a.W * plan.wrow_bytes;
+  plan.sign_bytes += (64u + 128u - plan.sign_bytes % 128u) % 128u;  // (64 mod 128; a multiple of 8 stays one)
+  plan.coin_off = plan.sign_bytes + (uint32_t)a.W * plan.wrow_bytes;
+  plan.rot_groups = c.rot_groups;
+  plan.probe = a.tune.wait_limit != 0;
+  plan.wait_limit = plan.probe ? a.tune.wait_limit : kPackWaitLimit;
   struct Tag {};
-  cudaError_t e = ensure_dynamic_smem<Tag>(decode_pack_kernel<NW, SIMPLE>, di.ordinal, c.smem);
+  cudaError_t e = ensure_dynamic_smem<Tag>(decode_pack_kernel<NW, SIMPLE, ROT>, di.ordinal, c.smem);
   if (e != cudaSuccess) return e;
   int64_t grid = di.sms;
   const int64_t need = (plan.n_items + c.warps - 1) / c.warps;
   if (grid > need) grid = need;
-  decode_pack_kernel<NW, SIMPLE><<<(unsigned)grid, c.warps * 32, c.smem, stream>>>(a, tab, plan);
+  decode_pack_kernel<NW, SIMPLE, ROT><<<(unsigned)grid, c.warps * 32, c.smem, stream>>>(a, tab, plan);
   count_launch();
   return cudaGetLastError();
 }
@@ -414,8 +557,11 @@ cudaError_t dispatch_nw(const DecodeArgs& a, const DecodeTables& tab, const Pack
     return cudaErrorInvalidValue;
   } else {
     if (c.nw == NW) {
-      if (c.nch == 1 && NW * 2 == a.C) return launch_pack<NW, true>(a, tab, c, di, stream);
-      return launch_pack<NW, false>(a, tab, c, di, stream);
+      if (c.nch == 1 && NW * 2 == a.C) {
+        if (c.rot_groups != 0) return launch_pack<NW, true, true>(a, tab, c, di, stream);
+        return launch_pack<NW, true, false>(a, tab, c, di, stream);
+      }
+      return launch_pack<NW, false, false>(a, tab, c, di, stream);
     }
     return dispatch_nw<NW + 1>(a, tab, c, di, stream);
   }
@@ -432,7 +578,7 @@ bool decode_pack_eligible(const DecodeArgs& a) {
   if (a.tune.kernel != 0 && a.tune.kernel != 4) return false;
   if (a.tune.kernel == 0 && (a.C < 6 || a.C > 2 * kPackMaxNW || a.G * (int64_t)a.W * a.C * 4 < (int64_t(64) << 20))) return false;
   if (a.y_rs != a.C || a.y_gs != (int64_t)a.W * a.C || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
-  if (!aligned16(a.Yt) || !aligned16(a.Yh)) return false;
+  if (!aligned16(a.Yt) || !aligned16(a.Yh) || !aligned16(a.mask)) return false;
   const DeviceInfo* di = nullptr;
   if (current_device_info(&di) != cudaSuccess) return false;
   PackChoice c;

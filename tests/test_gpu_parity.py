@@ -480,6 +480,10 @@ PACK_SHAPES = [
     (12, 20, 10, 999),    # six lanes per group: five groups do not start on 16-byte boundaries, four do
     (8, 24, 10, 333),
     (16, 24, 10, 1000),
+    (3, 7, 10, 50),       # coincident nodes with one lane per row (where the rotated word order can apply)
+    (5, 11, 10, 203),     # ... and three lanes per group, a ragged last item
+    (8, 12, 8, 100),      # rows of four words, every group starting in the same banks
+    (4, 8, 10, 333),      # two lanes per group, rotated because shared memory bounds it
 ]
 
 
@@ -487,8 +491,8 @@ PACK_SHAPES = [
 def test_packed_groups_decoder_against_oracle_and_register_decoder(K, W, C, G):
     """Dense buffers with an even number of classes up to 62 take the kernel in which every warp runs its own
     pipeline over items of several groups.  It adds the same terms in the same order as the per-column kernel:
-    equal to the last bit; absent rows (NaN here) never used; both sign rules; a two-slot ring with five warps
-    and a four-slot ring with one-group items forced as well."""
+    equal to the last bit; absent rows (NaN here) never used; both sign rules; five warps per CTA, one-group items,
+    and the rotated word order forced off and on as well."""
     rng = np.random.default_rng(K * 1000 + C)
     Yt = torch.randn((G, W, C), generator=torch.Generator().manual_seed(C + K))
     mask = random_masks(W, G, rng, min_present=0)
@@ -505,7 +509,8 @@ def test_packed_groups_decoder_against_oracle_and_register_decoder(K, W, C, G):
     for flags in (0, binding.SIGN_WORKER_INDEX):
         p = ap.make_params(K, W, 0, flags)
         ref = ap.approxifer_decode(p, dY, dm, tuning=ap.decode_tuning(kernel=1))
-        for tuning in (None, ap.decode_tuning(4, 2, 5, 0, 0), ap.decode_tuning(4, 4, 0, 1, 0)):
+        for tuning in (None, ap.decode_tuning(4, 2, 5, 0, 0), ap.decode_tuning(4, 4, 0, 1, 0),
+                       ap.decode_tuning(4, 0, 0, 0, 1), ap.decode_tuning(4, 0, 0, 0, 2)):
             n_used = torch.empty(G, dtype=torch.int32, device=dev())
             status = torch.empty(G, dtype=torch.int32, device=dev())
             guard = torch.full((G * K * C + 64,), CANARY, device=dev())
