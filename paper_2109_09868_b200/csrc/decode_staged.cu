@@ -118,8 +118,13 @@ constexpr int kTableOff = 128;  // float rg[W][K] after the mbarriers and the ab
 __host__ __device__ constexpr int slots_off(int W, int K) { return (kTableOff + W * (K | 1) * 4 + 127) / 128 * 128; }
 // (cb: bytes of a column of four elements -- 16 for fp32 payloads, 8 for bfloat16)
 __host__ __device__ constexpr int slot_bytes(int W, int KT, int SPLIT, int COLS, int cb = 16) { return meta_bytes(W, KT, SPLIT) + W * COLS * cb; }
+// Resident CTAs per SM the kernel is compiled and launched for.  The 96-thread configuration (rows of 17 .. 32
+// columns: C = 68 .. 128) runs 8 per SM with up to 6 queries per thread (measured 1.19-1.30x over 6: its items are
+// small and what hides their latency is more warps); with 7 or 8 queries per thread the registers that 8, or 7,
+// CTAs leave cost more than the extra warps gain (0.9x), and 12 CTAs of 64 threads or 5 of 160 changed nothing or
+// lost 2 %.
 __host__ __device__ constexpr int min_ctas(int KT, int threads) {
-  return KT > 8 ? 1 : (threads <= 64 ? 10 : (threads <= 96 ? 6 : (threads <= 160 ? 4 : (threads <= 288 ? 2 : 1))));
+  return KT > 8 ? 1 : (threads <= 64 ? 10 : (threads <= 96 ? (KT <= 6 ? 8 : 6) : (threads <= 160 ? 4 : (threads <= 288 ? 2 : 1))));
 }
 
 // Shared memory: full[4] empty[4] mbarriers, abort flag | rg[W][K] | S slots, each = item block + W rows of COLS*16 B.
@@ -410,8 +415,7 @@ cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t
   if (e != cudaSuccess) return e;
   const int sms = di->sms, smem_sm = di->smem_per_sm;
   const int fixed = slots_off(a.W, a.K);
-  // as many CTAs per SM as fit with a two-slot ring (at most 4 small or 2 large ones), then the ring as deep
-  // as the rest allows
+  // as many CTAs per SM as fit with a two-slot ring (up to min_ctas), then the ring as deep as the rest allows
   int ctas = min_ctas(KT, SPLIT * COLS + 32);
   if (a.tune.ctas_per_sm > 0 && a.tune.ctas_per_sm < ctas) ctas = a.tune.ctas_per_sm;
   while (ctas > 1 && (int64_t)ctas * (fixed + 2 * slot + 1024) > smem_sm) --ctas;
