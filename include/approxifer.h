@@ -381,6 +381,22 @@ int approxifer_debug_locate(const approxifer_params* params, int64_t G, int64_t 
                             int force_warp_kernel, void* cuda_stream);
 
 /*
+ * Host-side planning hook (no device call; the paper has no counterpart).  The packed-groups decoder keeps the
+ * predictions of several consecutive groups in shared memory exactly as they lie in device memory, so groups can
+ * start in the same banks; where that costs, some groups of a work item take the words of their rows in an
+ * order rotated by one.  Which ones is decided on the host from a model of the bank rules (a 64-bit load costs
+ * the largest number of different words that meet in one bank over the warp; a store the same per half-warp).
+ * For the shape (K, W, C) this returns the groups per work item (0: the kernel does not take the shape), the
+ * rotated groups as a bit set (bit s = group s of the item), and the model's count of shared-memory passes per
+ * item for the loads of the worker loop plus the stores of the results, without any rotation and with the chosen
+ * one (both 0 where rows are shared by several lanes and no rotation applies).  mode: 0 as the decoder decides,
+ * 1 never rotate, 2 rotate whenever the model prefers a set.  All pointers HOST, all required.
+ * APPROXIFER_E_PARAM for a null pointer or parameters outside 1 <= K <= W <= 32, C >= 1, mode in 0..2.
+ */
+int approxifer_debug_pack_rotation(int32_t K, int32_t W, int64_t C, int32_t mode, int32_t* groups_per_item,
+                                   uint32_t* rotated_groups, int32_t* passes_plain, int32_t* passes_chosen);
+
+/*
  * Measuring hook (not on the hot path; the paper has no counterpart): `blocks` CTAs of 256 threads each run
  * `iters` rounds of 64 dependent-chain-free fp32 multiply-adds per thread on registers only (16 independent
  * chains), 2 * 64 * iters * 256 * blocks flop in all.  Timed by the caller, it gives the issue rate of the plain

@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     approxifer_decode_tuning,
     decode_tuning,
     debug_fma_peak,
+    debug_pack_rotation,
     device_wait_timeouts,
     reset_device_wait_timeouts,
     launch_count,

@@ -44,6 +44,7 @@ EXPORTS = (
     "approxifer_locate_host",
     "approxifer_encode_host_static",
     "approxifer_debug_fma_peak",
+    "approxifer_debug_pack_rotation",
     "approxifer_encode_scatter",
     "approxifer_decode_gather",
     "approxifer_locate_gather",
@@ -129,6 +130,10 @@ def load() -> ctypes.CDLL:
     lib.approxifer_reset_device_wait_timeouts.restype = c_int
     lib.approxifer_debug_fma_peak.argtypes = [c_int, c_int, c_void_p, c_void_p]
     lib.approxifer_debug_fma_peak.restype = c_int
+    lib.approxifer_debug_pack_rotation.argtypes = [ctypes.c_int32, ctypes.c_int32, c_int64, ctypes.c_int32,
+                                                   POINTER(ctypes.c_int32), POINTER(ctypes.c_uint32),
+                                                   POINTER(ctypes.c_int32), POINTER(ctypes.c_int32)]
+    lib.approxifer_debug_pack_rotation.restype = c_int
     lib.approxifer_debug_locate.argtypes = [pp, c_int64, c_int64, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p,
                                             c_void_p, c_int, c_void_p]
     lib.approxifer_debug_locate.restype = c_int
@@ -173,6 +178,18 @@ def debug_fma_peak(iters: int, blocks: int, sink: torch.Tensor, stream=None) -> 
     rc = load().approxifer_debug_fma_peak(int(iters), int(blocks), sink.data_ptr(), _stream_ptr(stream))
     if rc != OK:
         raise ApproxiferError(rc, "approxifer_debug_fma_peak")
+
+
+def debug_pack_rotation(K: int, W: int, C: int, mode: int = 0):
+    """Host-side plan of the packed-groups decoder for a shape (no device call): (groups per work item, rotated
+    groups as a bit set, modelled shared-memory passes per item without rotation, with the chosen one)."""
+    gw, rot = ctypes.c_int32(0), ctypes.c_uint32(0)
+    plain, chosen = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = load().approxifer_debug_pack_rotation(int(K), int(W), int(C), int(mode), ctypes.byref(gw), ctypes.byref(rot),
+                                               ctypes.byref(plain), ctypes.byref(chosen))
+    if rc != OK:
+        raise ApproxiferError(rc, "approxifer_debug_pack_rotation")
+    return gw.value, rot.value, plain.value, chosen.value
 
 
 def device_wait_timeouts() -> int:

@@ -294,6 +294,18 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
                                         static_cast<cudaStream_t>(cuda_stream)));
 }
 
+int approxifer_debug_pack_rotation(int32_t K, int32_t W, int64_t C, int32_t mode, int32_t* groups_per_item,
+                                   uint32_t* rotated_groups, int32_t* passes_plain, int32_t* passes_chosen) {
+  if (groups_per_item == nullptr || rotated_groups == nullptr || passes_plain == nullptr || passes_chosen == nullptr)
+    return APPROXIFER_E_PARAM;
+  if (K < 1 || W < 2 || K > W || W > kMaxW || C < 1 || mode < 0 || mode > 2) return APPROXIFER_E_PARAM;
+  int gw = 0, plain = 0, chosen = 0;
+  uint32_t rot = 0;
+  if (!pack_rotation_info(K, W, C, mode, &gw, &rot, &plain, &chosen)) gw = 0, rot = 0, plain = 0, chosen = 0;
+  *groups_per_item = gw, *rotated_groups = rot, *passes_plain = plain, *passes_chosen = chosen;
+  return APPROXIFER_OK;
+}
+
 int approxifer_debug_fma_peak(int iters, int blocks, float* sink, void* cuda_stream) {
   if (iters < 1 || blocks < 1 || blocks > (1 << 20)) return APPROXIFER_E_RANGE;
   if (sink == nullptr) return APPROXIFER_E_NULL;

@@ -104,6 +104,8 @@ cudaError_t read_decode_wait_timeouts(unsigned int* out);
 bool decode_pack_eligible(const DecodeArgs& a);
 cudaError_t launch_decode_pack(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t stream);
 cudaError_t read_pack_wait_timeouts(unsigned int* out);
+bool pack_rotation_info(int K, int W, int64_t C, int mode, int* groups_per_item, uint32_t* rotated_groups,
+                        int* passes_plain, int* passes_chosen);
 cudaError_t reset_decode_wait_timeouts();
 cudaError_t reset_pack_wait_timeouts();
 

@@ -585,6 +585,25 @@ bool decode_pack_eligible(const DecodeArgs& a) {
   return plan_pack(a, di->smem_per_sm, &c);
 }
 
+// The plan's host-side choices for a shape, without a device: groups per item, the rotated groups, and the model's
+// shared-memory passes per item (loads of the worker loop + stores of the results) without and with them.
+bool pack_rotation_info(int K, int W, int64_t C, int mode, int* groups_per_item, uint32_t* rotated_groups,
+                        int* passes_plain, int* passes_chosen) {
+  DecodeArgs a{};
+  a.K = K, a.W = W, a.C = C, a.G = int64_t(1) << 30;
+  a.tune.split = mode;
+  PackChoice c;
+  if (!plan_pack(a, 227 * 1024, &c)) return false;
+  *groups_per_item = c.gw;
+  *rotated_groups = c.rot_groups;
+  *passes_plain = *passes_chosen = 0;
+  if (c.nch == 1 && c.nw * 2 == C) {
+    (void)rotation_cost(K, W, (int)C, c.gw, c.jt, 0u, passes_plain);
+    (void)rotation_cost(K, W, (int)C, c.gw, c.jt, c.rot_groups, passes_chosen);
+  }
+  return true;
+}
+
 cudaError_t reset_pack_wait_timeouts() {
   const unsigned int zero = 0;
   return cudaMemcpyToSymbol(g_pack_wait_timeouts, &zero, sizeof(unsigned int));
