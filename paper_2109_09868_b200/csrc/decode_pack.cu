@@ -570,13 +570,14 @@ cudaError_t dispatch_nw(const DecodeArgs& a, const DecodeTables& tab, const Pack
 }  // namespace
 
 // Dense buffers (rows and groups back to back), 16-byte aligned, an even number of classes up to 62.  Chosen
-// automatically where it is the fastest of the decoders (measured on 2 GB problems, K = 4 .. 16: 1.25-1.3x the
-// thread-per-(query, chunk) kernel at C = 10): rows of 6 .. 10 classes, which one lane covers whole, and
-// problems beyond the L2 cache (on cache-resident ones the two are equal and launch-bound).  Other even C up
-// to 62 run correctly when asked for (tuning kernel = 4) but lose to the other kernels.
+// automatically where it is the fastest of the decoders (measured on 3 GB problems, K = 4 .. 16: 1.1-1.5x the
+// thread-per-(query, chunk) kernel at C = 10): rows of 6 .. 10 classes, which one lane covers whole, and at
+// least 32 MB of predictions (K = 8, W = 12, C = 10: equal and launch-bound up to 65,536 groups, 1.10x at
+// 131,072, 1.26x at 524,288).  Other even C up to 62 run correctly when asked for (tuning kernel = 4); there the
+// other kernels are as fast or faster except at isolated C (32, 40, 62 with K <= 8).
 bool decode_pack_eligible(const DecodeArgs& a) {
   if (a.tune.kernel != 0 && a.tune.kernel != 4) return false;
-  if (a.tune.kernel == 0 && (a.C < 6 || a.C > 2 * kPackMaxNW || a.G * (int64_t)a.W * a.C * 4 < (int64_t(64) << 20))) return false;
+  if (a.tune.kernel == 0 && (a.C < 6 || a.C > 2 * kPackMaxNW || a.G * (int64_t)a.W * a.C * 4 < (int64_t(32) << 20))) return false;
   if (a.y_rs != a.C || a.y_gs != (int64_t)a.W * a.C || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
   if (!aligned16(a.Yt) || !aligned16(a.Yh) || !aligned16(a.mask)) return false;
   const DeviceInfo* di = nullptr;
