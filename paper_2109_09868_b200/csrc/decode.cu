@@ -229,7 +229,9 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
   if (a.G == 0) return cudaSuccess;
   const DecodeTables& tab = decode_tables(a.K, a.W);
   bool by4 = a.C % 4 == 0 && a.y_gs % 4 == 0 && (a.rows.on || a.y_rs % 4 == 0) && a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
-  if (a.rows.on) {  // gathered rows: the per-column kernel follows the offset table
+  if (a.rows.on) {  // gathered rows: the packed-groups kernel where it takes the shape, else the per-column kernel
+                    // follows the offset table
+    if (!a.bf16 && decode_pack_eligible(a)) return launch_decode_pack(a, tab, stream);
     for (int i = 0; i < a.W; ++i) by4 = by4 && a.rows.off[i] % 4 == 0;
     if (by4 && aligned16(a.Yt) && aligned16(a.Yh)) return dispatch_k<PayloadF32x4>(a, tab, stream);
     return dispatch_k<PayloadF32>(a, tab, stream);

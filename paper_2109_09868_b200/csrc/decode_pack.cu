@@ -1,6 +1,7 @@
 // ApproxIFER decoder for short payloads in dense buffers (Section 3, "Decoding", step 2): predictions of an even
 // number of classes up to 62 -- the paper's own workloads have C = 10 -- stored back to back ([G][W][C] in,
-// [G][K][C] out).
+// [G][K][C] out), or one batch per worker ([W][G][C], or W buffers of [G][C] given by a table of offsets: the
+// form in which the workers' answers arrive).
 //
 // Same arithmetic as decode_kernel, term by term and rounding by rounding (barycentric numerator and
 // denominator over the present workers in ascending order, one reciprocal per query), different data movement
@@ -12,7 +13,9 @@
 //    bulk asynchronous copies, one item ahead of the one being reduced (the ring has two slots: deeper rings
 //    measured slower, and cost registers), completion counted on one mbarrier per slot; a slot is refilled by the warp that has just finished reading it, so there are no "empty"
 //    barriers, no producer warp and no CTA-wide barrier in the main loop.  With a dozen such warps per SM
-//    there are always tens of KB of loads in flight and always some warp with arithmetic to do.
+//    there are always tens of KB of loads in flight and always some warp with arithmetic to do.  With one batch
+//    per worker an item is W pieces (a worker's rows of the item's groups), copied by W lanes, one piece each,
+//    onto the same mbarrier; inside the slot the rows then lie worker by worker.
 //  * Lane = (group of the item, tile of two queries, word lane).  A thread forms two queries for NW words
 //    (pairs of adjacent classes): every payload word it loads from shared memory feeds two packed
 //    multiply-adds (fma.rn.f32x2: both halves ordinary round-to-nearest fp32 FMAs), and the signed weights
@@ -117,6 +120,8 @@ struct PackPlan {
   // sizes the kernel would otherwise keep in registers (as kernel parameters they are read where they are used)
   uint32_t row_bytes;      // C floats
   uint32_t group_bytes;    // W rows
+  uint32_t y_group_step;   // bytes between two groups' rows of one worker inside a ring slot
+  uint32_t y_row_step;     // ... between two workers' rows of one group
   uint32_t result_bytes;   // K rows
   uint32_t wrow_bytes;     // one worker's row of the weight table: KP entries of 8 bytes
   uint32_t sign_bytes;     // between the two signs of the weight table (padded: the two copies of a row sit in
@@ -135,7 +140,7 @@ __device__ __forceinline__ float p_hi(uint64_t v) { return __uint_as_float((uint
 // wtab[sg][i][j] = (w, w) with w = (-1)^sg / (alpha_j - beta_i): the signed weight, already duplicated for the
 // packed multiply-add (the sign flip is exact, so (s rg) y rounds like rg (s y)).
 // SIMPLE: one lane owns all the words of its rows (nch == 1, NW == C/2), so every offset is a compile-time constant.
-template <int NW, bool SIMPLE, bool ROT>
+template <int NW, bool SIMPLE, bool ROT, bool WM>
 __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     decode_pack_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ DecodeTables tab,
                        const __grid_constant__ PackPlan plan) {
@@ -177,7 +182,7 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
   const int Cw = C >> 1;
   const bool exact = SIMPLE || NW * nch == Cw;  // no lane has a word beyond the end of the row
   const bool literal = (a.flags & kFlagSignWorkerIndex) != 0;
-  const uint32_t y_off = (uint32_t)s * plan.group_bytes + (uint32_t)ch * 8u;
+  const uint32_t y_off = (uint32_t)s * plan.y_group_step + (uint32_t)ch * 8u;
   const uint32_t o_off = (uint32_t)(s * K + j0) * plan.row_bytes + (uint32_t)ch * 8u;
   const uint32_t u_step = (uint32_t)nch * 8u;
   // Where register slot u's word sits in a row.  With one lane per row (SIMPLE) the groups whose rows start in the
@@ -193,35 +198,53 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
   const int c0 = (j0 < K) ? coins[j0] : -1, c1 = (j0 + 1 < K) ? coins[j0 + 1] : -1;
   const unsigned char* wrow0 = reinterpret_cast<const unsigned char*>(wtab) + (uint32_t)j0 * 8u;
 
-  // lane 0: start the copy of the item whose first group is g0 into ring slot `slot`.  A ragged last item may end
-  // on an 8-byte boundary: the copy takes the whole 16-byte columns and the last two floats go by hand.
+  // Start the copies of the item whose first group is g0 into ring slot `slot`.  Group-major predictions (called
+  // by lane 0): one copy of the whole block; a ragged last item may end on an 8-byte boundary: the copy takes the
+  // whole 16-byte columns and the last two floats go by hand.  Worker-major (WM; called by the whole warp): lane 0
+  // announces the bytes, lane i starts the copy of worker i's rows of the item's groups, which land worker by
+  // worker, GW rows apart; a last item whose pieces are not whole 16-byte columns goes by hand.
   auto issue = [&](int64_t g0, int slot) {
     const int ng = (int)min((int64_t)GW, a.G - g0);
-    const uint32_t bytes = (uint32_t)ng * plan.group_bytes, bytes16 = bytes & ~15u;
-    const unsigned char* src = reinterpret_cast<const unsigned char*>(a.Yt) + g0 * (int64_t)plan.group_bytes;
     unsigned char* dst = slots + (size_t)slot * plan.in_bytes;
     const uint32_t bar = p_smem_u32(full + slot);
     // (test hook: the item that holds one chosen group is never fetched, so the wait for it runs out)
     if (a.tune.withhold_group >= g0 && a.tune.withhold_group < g0 + ng) return;
-    if (bytes16 != bytes) *reinterpret_cast<float2*>(dst + bytes16) = *reinterpret_cast<const float2*>(src + bytes16);
     // the item's masks travel the same way: the whole 16-byte columns of the mask array that hold them (group g's
     // mask lands at word (g0 & 3) + g - g0 of the slot's mask area); by hand where those would end beyond the array
     const int64_t m0 = g0 & ~int64_t(3), m1 = (g0 + ng + 3) & ~int64_t(3);
-    uint32_t mask_bytes = 0;
-    if (m1 <= a.G) mask_bytes = (uint32_t)(m1 - m0) * 4u;
-    else
+    const uint32_t mask_bytes = m1 <= a.G ? (uint32_t)(m1 - m0) * 4u : 0u;
+    if (lane == 0 && mask_bytes == 0)
       for (int q = 0; q < ng; ++q) reinterpret_cast<uint32_t*>(dst + plan.mask_off)[(int)(g0 & 3) + q] = a.mask[g0 + q];
-    // (release: what was written by hand above is visible to whoever sees the phase complete)
-    p_arrive_expect_tx(bar, bytes16 + mask_bytes);
-    if (bytes16) p_bulk_g2s(p_smem_u32(dst), src, bytes16, bar);
-    if (mask_bytes) p_bulk_g2s(p_smem_u32(dst + plan.mask_off), a.mask + m0, mask_bytes, bar);
+    if constexpr (!WM) {
+      const uint32_t bytes = (uint32_t)ng * plan.group_bytes, bytes16 = bytes & ~15u;
+      const unsigned char* src = reinterpret_cast<const unsigned char*>(a.Yt) + g0 * (int64_t)plan.group_bytes;
+      if (bytes16 != bytes) *reinterpret_cast<float2*>(dst + bytes16) = *reinterpret_cast<const float2*>(src + bytes16);
+      // (release: what was written by hand above is visible to whoever sees the phase complete)
+      p_arrive_expect_tx(bar, bytes16 + mask_bytes);
+      if (bytes16) p_bulk_g2s(p_smem_u32(dst), src, bytes16, bar);
+      if (mask_bytes) p_bulk_g2s(p_smem_u32(dst + plan.mask_off), a.mask + m0, mask_bytes, bar);
+    } else {
+      const uint32_t piece = (uint32_t)ng * plan.row_bytes;  // one worker's rows of the item's groups
+      const bool whole = (piece & 15u) == 0;
+      const float* src = a.Yt + (a.rows.on ? a.rows.off[lane < W ? lane : 0] : (int64_t)lane * a.y_rs) + g0 * (int64_t)C;
+      unsigned char* mine_dst = dst + (uint32_t)lane * plan.y_row_step;
+      if (!whole && lane < W)
+        for (uint32_t f = 0; f < piece / 4u; ++f) reinterpret_cast<float*>(mine_dst)[f] = src[f];
+      __syncwarp();  // (what the lanes wrote by hand is ordered before lane 0's release below)
+      if (lane == 0) {
+        p_arrive_expect_tx(bar, (whole ? (uint32_t)W * piece : 0u) + mask_bytes);
+        if (mask_bytes) p_bulk_g2s(p_smem_u32(dst + plan.mask_off), a.mask + m0, mask_bytes, bar);
+      }
+      if (whole && lane < W) p_bulk_g2s(p_smem_u32(mine_dst), src, piece, bar);
+    }
   };
+
   const bool probe = plan.probe != 0;  // (test hook: a short limit, counted in non-blocking probes)
   // prologue: one item in flight
   const int64_t g_stride = stride * GW;
   int left = (int)my_items;  // items this warp has still to reduce (the launch keeps this below 2^31)
   int64_t g0 = first * GW;   // first group of the item being reduced
-  if (lane == 0 && left > 0) issue(g0, 0);
+  if ((WM || lane == 0) && left > 0) issue(g0, 0);
 
   int slot = 0;  // ring slot of the item being reduced; the item started in the same iteration goes to the other
   uint32_t parity = 0;
@@ -230,7 +253,7 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     const int ng = (int)min((int64_t)GW, a.G - g0);
     // the slot that the previous item occupied is free (its results were copied out of it before the __syncwarp
     // that ended the previous iteration): refill it with the next item
-    if (lane == 0 && left > 1) issue(g0 + g_stride, slot ^ 1);
+    if ((WM || lane == 0) && left > 1) issue(g0 + g_stride, slot ^ 1);
     // wait for this item's bytes (bounded)
     {
       const uint32_t addr = p_smem_u32(full + slot);
@@ -264,7 +287,7 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
       const unsigned char* yr = yg;
       const unsigned char* wr = wrow0;
 #pragma unroll 2
-      for (int i = 0; i < W; ++i, yr += plan.row_bytes, wr += plan.wrow_bytes) {
+      for (int i = 0; i < W; ++i, yr += plan.y_row_step, wr += plan.wrow_bytes) {
         uint64_t y[NW];
 #pragma unroll
         for (int u = 0; u < NW; ++u) {  // (an absent worker's row may be loaded; it is only used under `present`)
@@ -292,8 +315,8 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
 #pragma unroll
         for (int u = 0; u < NW; ++u) {
           if (exact || u * nch + ch < Cw) {
-            if (pin0) acc0[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c0 * plan.row_bytes + woff(u));
-            if (pin1) acc1[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c1 * plan.row_bytes + woff(u));
+            if (pin0) acc0[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c0 * plan.y_row_step + woff(u));
+            if (pin1) acc1[u] = *reinterpret_cast<const uint64_t*>(yg + (uint32_t)c1 * plan.y_row_step + woff(u));
           }
         }
       }
@@ -348,6 +371,7 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
 struct PackChoice {
   int nw = 0, nch = 0, jt = 0, gw = 0, warps = 0;
   uint32_t rot_groups = 0;
+  bool worker_major = false;
   int in_bytes = 0, mask_off = 0, table_bytes = 0, smem = 0;
 };
 
@@ -382,9 +406,10 @@ void choose_words(int Cw, int* nw, int* nch) {
 // move across sets with the same number of passes).  A pass of a store counts twice: the stores sit in the
 // dependent tail of an item, between two warp barriers, and measured about that much dearer than the loads of
 // the pipelined worker loop.
-int64_t rotation_cost(int K, int W, int C, int gw, int jt, uint32_t rot_groups, int* passes = nullptr) {
+// in_step: bytes between two groups' rows of one worker in a ring slot (W C 4 group-major, C 4 worker-major).
+int64_t rotation_cost(int K, int W, int C, int gw, int jt, uint32_t in_step, uint32_t rot_groups, int* passes = nullptr) {
   const int NW = C / 2;
-  const uint32_t row_bytes = (uint32_t)C * 4u, group_bytes = (uint32_t)W * row_bytes, result_bytes = (uint32_t)K * row_bytes;
+  const uint32_t row_bytes = (uint32_t)C * 4u, group_bytes = in_step, result_bytes = (uint32_t)K * row_bytes;
   int loads = 0, stores = 0, excess_loads = 0, excess_stores = 0;
   for (int u = 0; u < NW; ++u) {
     uint32_t seen[16][32];  // the different words met so far in each bank pair
@@ -439,35 +464,35 @@ int64_t rotation_cost(int K, int W, int C, int gw, int jt, uint32_t rot_groups, 
 // DRAM rate, and the rotated code has a few more instructions); rows of fewer than 8 classes lost either way.
 // The answer depends on the shape alone and is remembered per shape.  mode (tuning): 1 never, 2 whenever the
 // model prefers a set.
-uint32_t choose_rotation(int K, int W, int C, int gw, int jt, int mode) {
+uint32_t choose_rotation(int K, int W, int C, int gw, int jt, uint32_t in_step, int mode) {
   if (mode == 1 || gw < 2) return 0u;
   struct Entry {
     int K, W, C, gw, mode;
-    uint32_t rot;
+    uint32_t in_step, rot;
   };
   static std::mutex mu;
   static std::vector<Entry> memo;
   {
     std::lock_guard<std::mutex> lock(mu);
     for (const Entry& e : memo)
-      if (e.K == K && e.W == W && e.C == C && e.gw == gw && e.mode == mode) return e.rot;
+      if (e.K == K && e.W == W && e.C == C && e.gw == gw && e.mode == mode && e.in_step == in_step) return e.rot;
   }
   int plain_passes = 0;
-  const int64_t plain = rotation_cost(K, W, C, gw, jt, 0u, &plain_passes);
+  const int64_t plain = rotation_cost(K, W, C, gw, jt, in_step, 0u, &plain_passes);
   uint32_t best = 0u;
   int64_t best_cost = plain;
   for (uint32_t m = 1; m < 32; ++m) {
     uint32_t cand = 0u;
     for (int s = 0; s < gw; ++s)
       if (__builtin_popcount((uint32_t)s & m) & 1) cand |= 1u << s;
-    const int64_t c = rotation_cost(K, W, C, gw, jt, cand);
+    const int64_t c = rotation_cost(K, W, C, gw, jt, in_step, cand);
     if (c < best_cost) best = cand, best_cost = c;
   }
   for (int round = 0; round < 3; ++round) {
     bool changed = false;
     for (int s = 0; s < gw; ++s) {
       const uint32_t cand = best ^ (1u << s);
-      const int64_t c = rotation_cost(K, W, C, gw, jt, cand);
+      const int64_t c = rotation_cost(K, W, C, gw, jt, in_step, cand);
       if (c < best_cost) best = cand, best_cost = c, changed = true;
     }
     if (!changed) break;
@@ -480,13 +505,26 @@ uint32_t choose_rotation(int K, int W, int C, int gw, int jt, int mode) {
   const bool use = best_cost < plain && (mode == 2 || (C >= 8 && (jt >= 3 || bound_by_shared)));
   const uint32_t rot = use ? best : 0u;
   std::lock_guard<std::mutex> lock(mu);
-  if (memo.size() < 256) memo.push_back(Entry{K, W, C, gw, mode, rot});
+  if (memo.size() < 256) memo.push_back(Entry{K, W, C, gw, mode, in_step, rot});
   return rot;
+}
+
+// One batch per worker: rows of a worker C apart from group to group, the workers' batches anywhere (a table of
+// offsets, or a stride that keeps them apart), all on 16-byte boundaries.
+bool pack_worker_major(const DecodeArgs& a) {
+  if (a.y_gs != a.C) return false;
+  if (a.rows.on) {
+    for (int i = 0; i < a.W; ++i)
+      if (a.rows.off[i] % 4 != 0) return false;
+    return true;
+  }
+  return a.y_rs % 4 == 0 && a.y_rs >= a.G * a.C;
 }
 
 bool plan_pack(const DecodeArgs& a, int smem_per_sm, PackChoice* out) {
   PackChoice p;
   const int K = a.K, W = a.W, C = (int)a.C;
+  p.worker_major = !(a.y_rs == a.C && a.y_gs == (int64_t)a.W * a.C && !a.rows.on) && pack_worker_major(a);
   if (C < 2 || C > kPackMaxC || (C & 1)) return false;
   p.jt = (K + 1) / 2;
   choose_words(C / 2, &p.nw, &p.nch);
@@ -496,7 +534,9 @@ bool plan_pack(const DecodeArgs& a, int smem_per_sm, PackChoice* out) {
   if (a.tune.cols > 0 && a.tune.cols < gw) gw = a.tune.cols;  // (tuning: upper bound on the groups per item)
   if ((int64_t)gw > a.G) gw = (int)a.G;
   // every item, and its block of results, starts on a 16-byte boundary
-  while (gw >= 1 && (int64_t)gw < a.G && (((int64_t)gw * W * C) % 4 != 0 || ((int64_t)gw * K * C) % 4 != 0)) --gw;
+  // (worker-major: every worker's piece of an item)
+  const int in_unit = p.worker_major ? C : W * C;
+  while (gw >= 1 && (int64_t)gw < a.G && (((int64_t)gw * in_unit) % 4 != 0 || ((int64_t)gw * K * C) % 4 != 0)) --gw;
   if (gw < 1) return false;
   p.gw = gw;
   if (K > W) return false;  // (the results of an item are staged in the slot of its predictions)
@@ -515,13 +555,17 @@ bool plan_pack(const DecodeArgs& a, int smem_per_sm, PackChoice* out) {
   if (a.tune.ctas_per_sm > 0 && a.tune.ctas_per_sm < warps) warps = a.tune.ctas_per_sm;  // (tuning: warps per CTA)
   if (warps < 4) return false;
   p.warps = warps;
-  if (p.nch == 1 && p.nw * 2 == C) p.rot_groups = choose_rotation(K, W, C, gw, p.jt, a.tune.split);
+  // (worker-major items hold a worker's rows of consecutive groups back to back, C floats apart; there the
+  // sets the model prefers measured 0.91-0.93x -- what bounds that form is the W small copies per item, not
+  // shared memory -- so nothing is rotated)
+  if (p.nch == 1 && p.nw * 2 == C && !p.worker_major)
+    p.rot_groups = choose_rotation(K, W, C, gw, p.jt, (uint32_t)(W * C * 4), a.tune.split);
   p.smem = p.table_bytes + warps * per_warp;
   *out = p;
   return true;
 }
 
-template <int NW, bool SIMPLE, bool ROT>
+template <int NW, bool SIMPLE, bool ROT, bool WM>
 cudaError_t launch_pack(const DecodeArgs& a, const DecodeTables& tab, const PackChoice& c, const DeviceInfo& di,
                         cudaStream_t stream) {
   PackPlan plan;
@@ -531,6 +575,8 @@ cudaError_t launch_pack(const DecodeArgs& a, const DecodeTables& tab, const Pack
   const int KP = (a.K + 1) & ~1;
   plan.row_bytes = (uint32_t)a.C * 4u;
   plan.group_bytes = (uint32_t)a.W * plan.row_bytes;
+  plan.y_group_step = c.worker_major ? plan.row_bytes : plan.group_bytes;
+  plan.y_row_step = c.worker_major ? (uint32_t)c.gw * plan.row_bytes : plan.row_bytes;
   plan.result_bytes = (uint32_t)a.K * plan.row_bytes;
   plan.wrow_bytes = (uint32_t)KP * 8u;
   plan.sign_bytes = (uint32_t)a.W * plan.wrow_bytes;
@@ -540,12 +586,12 @@ cudaError_t launch_pack(const DecodeArgs& a, const DecodeTables& tab, const Pack
   plan.probe = a.tune.wait_limit != 0;
   plan.wait_limit = plan.probe ? a.tune.wait_limit : kPackWaitLimit;
   struct Tag {};
-  cudaError_t e = ensure_dynamic_smem<Tag>(decode_pack_kernel<NW, SIMPLE, ROT>, di.ordinal, c.smem);
+  cudaError_t e = ensure_dynamic_smem<Tag>(decode_pack_kernel<NW, SIMPLE, ROT, WM>, di.ordinal, c.smem);
   if (e != cudaSuccess) return e;
   int64_t grid = di.sms;
   const int64_t need = (plan.n_items + c.warps - 1) / c.warps;
   if (grid > need) grid = need;
-  decode_pack_kernel<NW, SIMPLE, ROT><<<(unsigned)grid, c.warps * 32, c.smem, stream>>>(a, tab, plan);
+  decode_pack_kernel<NW, SIMPLE, ROT, WM><<<(unsigned)grid, c.warps * 32, c.smem, stream>>>(a, tab, plan);
   count_launch();
   return cudaGetLastError();
 }
@@ -558,10 +604,12 @@ cudaError_t dispatch_nw(const DecodeArgs& a, const DecodeTables& tab, const Pack
   } else {
     if (c.nw == NW) {
       if (c.nch == 1 && NW * 2 == a.C) {
-        if (c.rot_groups != 0) return launch_pack<NW, true, true>(a, tab, c, di, stream);
-        return launch_pack<NW, true, false>(a, tab, c, di, stream);
+        if (c.worker_major) return launch_pack<NW, true, false, true>(a, tab, c, di, stream);
+        if (c.rot_groups != 0) return launch_pack<NW, true, true, false>(a, tab, c, di, stream);
+        return launch_pack<NW, true, false, false>(a, tab, c, di, stream);
       }
-      return launch_pack<NW, false, false>(a, tab, c, di, stream);
+      if (c.worker_major) return launch_pack<NW, false, false, true>(a, tab, c, di, stream);
+      return launch_pack<NW, false, false, false>(a, tab, c, di, stream);
     }
     return dispatch_nw<NW + 1>(a, tab, c, di, stream);
   }
@@ -569,7 +617,8 @@ cudaError_t dispatch_nw(const DecodeArgs& a, const DecodeTables& tab, const Pack
 
 }  // namespace
 
-// Dense buffers (rows and groups back to back), 16-byte aligned, an even number of classes up to 62.  Chosen
+// Dense buffers (rows and groups back to back, or one dense batch per worker), 16-byte aligned, an even number of
+// classes up to 62.  Chosen
 // automatically where it is the fastest of the decoders (measured on 3 GB problems, K = 4 .. 16: 1.1-1.5x the
 // thread-per-(query, chunk) kernel at C = 10): rows of 6 .. 10 classes, which one lane covers whole, and at
 // least 32 MB of predictions (K = 8, W = 12, C = 10: equal and launch-bound up to 65,536 groups, 1.10x at
@@ -578,7 +627,8 @@ cudaError_t dispatch_nw(const DecodeArgs& a, const DecodeTables& tab, const Pack
 bool decode_pack_eligible(const DecodeArgs& a) {
   if (a.tune.kernel != 0 && a.tune.kernel != 4) return false;
   if (a.tune.kernel == 0 && (a.C < 6 || a.C > 2 * kPackMaxNW || a.G * (int64_t)a.W * a.C * 4 < (int64_t(32) << 20))) return false;
-  if (a.y_rs != a.C || a.y_gs != (int64_t)a.W * a.C || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
+  const bool group_major = a.y_rs == a.C && a.y_gs == (int64_t)a.W * a.C && !a.rows.on;
+  if (!(group_major || pack_worker_major(a)) || a.o_rs != a.C || a.o_gs != (int64_t)a.K * a.C) return false;
   if (!aligned16(a.Yt) || !aligned16(a.Yh) || !aligned16(a.mask)) return false;
   const DeviceInfo* di = nullptr;
   if (current_device_info(&di) != cudaSuccess) return false;
@@ -599,8 +649,8 @@ bool pack_rotation_info(int K, int W, int64_t C, int mode, int* groups_per_item,
   *rotated_groups = c.rot_groups;
   *passes_plain = *passes_chosen = 0;
   if (c.nch == 1 && c.nw * 2 == C) {
-    (void)rotation_cost(K, W, (int)C, c.gw, c.jt, 0u, passes_plain);
-    (void)rotation_cost(K, W, (int)C, c.gw, c.jt, c.rot_groups, passes_chosen);
+    (void)rotation_cost(K, W, (int)C, c.gw, c.jt, (uint32_t)(W * C * 4), 0u, passes_plain);
+    (void)rotation_cost(K, W, (int)C, c.gw, c.jt, (uint32_t)(W * C * 4), c.rot_groups, passes_chosen);
   }
   return true;
 }

@@ -575,6 +575,40 @@ def test_short_payload_decoder_reads_worker_major_predictions(K, W, C, G):
     assert torch.equal(Yh.view(torch.int32), ref.view(torch.int32))
 
 
+@pytest.mark.parametrize("K,W,C,G", [(8, 12, 10, 1000), (8, 12, 10, 67), (4, 5, 10, 7), (5, 9, 10, 131), (3, 7, 10, 50),
+                                     (16, 24, 10, 333), (8, 12, 6, 100), (3, 7, 20, 50), (12, 20, 10, 999), (2, 4, 8, 260)])
+def test_packed_groups_decoder_reads_worker_major_predictions(K, W, C, G):
+    """The packed-groups kernel on predictions stored one batch per worker ([W][G][C]): an item's rows arrive by one
+    bulk copy per worker (by hand where a last item's pieces are not whole 16-byte columns).  Absent rows (NaN)
+    never used, both sign rules, coincident nodes ((3, 7)), bit-equal to the per-column kernel on the same view."""
+    rng = np.random.default_rng(K * 7 + C)
+    Yt = torch.randn((G, W, C), generator=torch.Generator().manual_seed(C + 3 * K))
+    mask = random_masks(W, G, rng, min_present=0)
+    mask[0] = 0
+    mask[G - 1] = 2**W - 1
+    dirty = Yt.clone()
+    for gi in range(G):
+        for i in range(W):
+            if not (int(mask[gi]) >> i) & 1:
+                dirty[gi, i] = float("nan")
+    wm = dirty.to(dev()).permute(1, 0, 2).contiguous()        # [W][G][C]
+    view = wm.permute(1, 0, 2)                                # [G][W][C] view: gstride = C, rstride = G*C
+    for flags in (0, binding.SIGN_WORKER_INDEX):
+        p = ap.make_params(K, W, 0, flags)
+        ref = ap.approxifer_decode(p, view, ap.mask_tensor(mask), tuning=ap.decode_tuning(kernel=1))
+        for tuning in (ap.decode_tuning(kernel=4), ap.decode_tuning(4, 0, 5, 3, 0)):
+            n_used = torch.empty(G, dtype=torch.int32, device=dev())
+            status = torch.empty(G, dtype=torch.int32, device=dev())
+            guard = torch.full((G * K * C + 64,), CANARY, device=dev())
+            Yh = guard[32: 32 + G * K * C].view(G, K, C)
+            ap.approxifer_decode(p, view, ap.mask_tensor(mask), Yh, n_used=n_used, status=status, tuning=tuning)
+            if flags == 0:
+                check_decode(K, W, Yt, mask, Yh, n_used, status, flags)
+            assert bool((guard[:32] == CANARY).all()) and bool((guard[32 + G * K * C:] == CANARY).all())
+            assert torch.equal(Yh.contiguous().view(torch.int32), ref.view(torch.int32))
+    assert ap.device_wait_timeouts() == 0
+
+
 @pytest.mark.parametrize("K,E,S,W,C", [(8, 2, 2, 24, 10), (3, 2, 1, 12, 37), (4, 1, 2, 12, 300), (2, 1, 0, 6, 1), (7, 3, 1, 22, 10),
                                        (10, 1, 0, 22, 10), (10, 2, 3, 27, 10), (12, 1, 0, 26, 10), (10, 3, 2, 28, 7), (11, 2, 6, 32, 10),
                                        (9, 2, 1, 23, 140), (12, 2, 0, 28, 10), (12, 3, 1, 31, 10), (13, 2, 2, 32, 5)])

@@ -61,6 +61,36 @@ def test_decode_gather_reads_every_present_worker_batch(K, W, G, C):
     assert torch.equal(Yh.view(torch.int32), ref.view(torch.int32))
 
 
+def test_decode_gather_beyond_the_cache_takes_the_packed_groups_kernel():
+    """80,000 groups of the paper's decode shape, one buffer per worker (38 MB in all): the automatic choice is the
+    packed-groups kernel reading each worker's rows through the offset table.  Bit-equal to the per-column kernel on
+    the same values stored group-major; a sample against the oracle."""
+    K, W, C, G = 8, 12, 10, 80000
+    rng = np.random.default_rng(11)
+    Yt = torch.randn((G, W, C), generator=torch.Generator().manual_seed(17))
+    mask = rng.integers(0, 2**W, size=G, dtype=np.uint64).astype(np.uint32)
+    mask[0], mask[1] = 0, 2**W - 1
+    rows = [Yt[:, i].clone().to(dev()) for i in range(W)]
+    p = ap.make_params(K, W)
+    n_used = torch.empty(G, dtype=torch.int32, device=dev())
+    status = torch.empty(G, dtype=torch.int32, device=dev())
+    launches = ap.launch_count()
+    Yh = ap.approxifer_decode_gather(p, rows, ap.mask_tensor(mask), n_used=n_used, status=status)
+    assert ap.launch_count() == launches + 1
+    ref = ap.approxifer_decode(p, Yt.to(dev()), ap.mask_tensor(mask), tuning=ap.decode_tuning(kernel=1))
+    assert torch.equal(Yh.view(torch.int32), ref.view(torch.int32))
+    n = 3000
+    want, n_ref, st_ref = oracle.decode(K, W, Yt[:n].numpy(), mask[:n])
+    got = Yh[:n].cpu().numpy().astype(np.float64)
+    scale = np.maximum(np.abs(want).reshape(n, -1).max(axis=1), 1e-30)
+    ok = np.isfinite(want).reshape(n, -1).all(axis=1)
+    err = np.abs(got - want).reshape(n, -1).max(axis=1)
+    assert np.all(err[ok] <= 1e-4 * scale[ok])
+    np.testing.assert_array_equal(n_used[:n].cpu().numpy(), n_ref)
+    np.testing.assert_array_equal(status[:n].cpu().numpy().view(np.uint32), st_ref)
+    assert ap.device_wait_timeouts() == 0
+
+
 @pytest.mark.parametrize("K,E,S,W,C", [(8, 2, 2, 24, 10), (4, 1, 1, 12, 37), (13, 3, 0, 32, 10)])
 def test_locate_gather_finds_the_same_workers(K, E, S, W, C):
     G = 120
