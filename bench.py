@@ -563,6 +563,11 @@ def other_workloads(ap, dev, peak):
     e["workload"] = "decode K=32 W=32 C=1000, all workers present"
     out.append(e)
     torch.cuda.empty_cache()
+    # the paper's own decode shape beyond the cache, predictions stored one batch per worker
+    e = synthetic_decode(ap, dev, 8, 12, 10, 3749888, worker_major=True)
+    e["workload"] = "decode K=8 W=12 C=10 on a 3 GB problem, predictions stored worker-major [W][G][C], 0-4 stragglers"
+    out.append(e)
+    torch.cuda.empty_cache()
     return out
 
 
