@@ -257,6 +257,11 @@ bool decode_small_eligible(const DecodeArgs& a) {
   // on the bulk-copy staged kernel takes over).
   // Elsewhere below 64 the per-column kernel is as fast or faster (both reach 3-3.5 TB/s there).
   if (!(a.C <= 36 || (a.K >= 14 && a.C < 64))) return false;
+  // ... except (measured on 1.5 GB problems, K = 4 .. 16; left to the per-column kernel unless this one is asked
+  // for): rows of 2 or 4 classes, where one 16-byte column per thread is already the whole row or half of it
+  // (per-column 1.1-1.8x), and rows of exactly 32 classes with K <= 12, where every row starts in the same
+  // shared-memory banks (per-column 1.2-1.7x).
+  if (a.tune.kernel == 0 && group_major && (a.C <= 4 || (a.C == 32 && a.K <= 12))) return false;
   return groups_per_cta(a, p) >= 1;
 }
 
