@@ -338,7 +338,7 @@ int approxifer_debug_weights(const approxifer_params* params, uint32_t mask, int
  *   kernel       1: route the call through the per-column register-staged kernel whatever the shape; 2, 3, 4: prefer
  *                the thread-per-(query, chunk) kernel, the bulk-copy staged kernel, the packed-groups kernel where
  *                that kernel takes the shape (else the automatic choice among the remaining ones)
- *   stages       bulk-copy staged kernel (rows of >= 64 floats on the 128-bit path): upper bound >= 2 on the ring depth
+ *   stages       bulk-copy staged kernel (rows of >= 64 floats, 52 with K >= 8, on the 128-bit path): upper bound >= 2 on the ring depth
  *   ctas_per_sm  ... upper bound on resident CTAs per SM
  *   cols         ... 16, 32 (split 2 only), 64, 128 or 256 16-byte columns per work item (256 needs split 1 or 2
  *                and a ring that fits in shared memory, else 128 is used)

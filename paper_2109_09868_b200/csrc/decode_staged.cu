@@ -437,6 +437,8 @@ cudaError_t launch_kt(const DecodeArgs& a, const DecodeTables& tab, cudaStream_t
 
 constexpr int kWholeMaxK = 16;  // most queries one thread forms (SPLIT = 1)
 constexpr int kStagedMinC = 64;
+constexpr int kStagedMinCManyQueries = 52;  // K >= 8: rows of 52 .. 60 floats too (2 GB problems: 1.12-1.36x the
+                                            // per-column kernel at K = 8, 12; with K = 4 it is 0.5x, below 52 it loses)
 
 // Columns per work item.  Long contiguous pieces are what HBM likes: with 256 columns an item of workload 4
 // (rows of 250 float4) is whole rows -- one 4000-byte copy per present worker instead of two copies of about 2 KB
@@ -489,7 +491,7 @@ cudaError_t dispatch_kt(int kt, const DecodeArgs& a, const DecodeTables& tab, cu
 
 }  // namespace
 
-// Rows of at least 64 floats on the 128-bit path (measured against the other two decoders on 3 GB problems,
+// Rows of at least 64 floats (52 with K >= 8) on the 128-bit path (measured against the other two decoders on 3 GB problems,
 // K = 8 .. 16: 3.6-4.9 TB/s at C = 64, 3.8-4.5 TB/s at C = 96-100, 5.0-5.7 TB/s at C = 128, 4.9-5.9 TB/s from
 // C = 200 on, where they reach 2.1-3.8 TB/s; at C = 40-48 they are as fast or faster).  Narrower payloads, and
 // the (K, W) pairs in which some alpha_j equals some beta_i (the row-copy case), stay on the other kernels.
@@ -499,7 +501,8 @@ bool decode_staged_eligible(const DecodeArgs& a) {
              a.o_gs % 4 == 0 && a.o_rs % 4 == 0;
   // bfloat16: a column of four elements is 8 bytes, and every bulk copy must start and end on 16-byte boundaries
   if (a.bf16) vec = vec && a.C % 8 == 0 && a.y_gs % 8 == 0 && a.y_rs % 8 == 0 && a.K <= kWholeMaxK;
-  if (!(vec && a.C >= kStagedMinC * (a.bf16 ? 2 : 1))) return false;
+  const int64_t min_c = (a.K >= 8 && !a.bf16) ? kStagedMinCManyQueries : kStagedMinC * (a.bf16 ? 2 : 1);
+  if (!(vec && a.C >= min_c)) return false;
   for (int j = 0; j < a.K; ++j)
     for (int i = 0; i < a.W; ++i)
       if (nodes_coincide(a.K, a.W, j, i)) return false;

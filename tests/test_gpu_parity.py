@@ -380,6 +380,8 @@ STAGED_SHAPES = [
     (8, 12, 70, 200, 0),      # 50 columns
     (12, 20, 33, 256, 0),     # exactly one 64-column item per group
     (16, 24, 40, 400, 0),     # 100 columns: 128-column items
+    (8, 12, 77, 52, 0),       # K >= 8: rows of 52 .. 60 floats too (13 of 16 columns in use)
+    (12, 20, 50, 60, 0),
 ]
 
 
