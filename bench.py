@@ -515,7 +515,7 @@ def other_workloads(ap, dev, peak):
     med, mn = time_launches(lambda: ap.approxifer_locate_gather(p5, rows5, mt), 3, 10)
     entry("configs[4] locate, predictions gathered from one buffer per worker (approxifer_locate_gather)", locate_bytes(w5, m5), med, mn, w5.G)
     med, mn = time_launches(lambda: ap.approxifer_decode_gather(p5, rows5, trusted, Yh), 3, 10)
-    entry("configs[4] decode from trusted, gathered from one buffer per worker (approxifer_decode_gather)", decode_bytes(w5, t5), med, mn, w5.G)
+    entry("configs[4] decode from trusted, gathered from one buffer per worker (approxifer_decode_gather; host-bound at this size: the binding checks W tensors per call, the kernel is the worker-major one above)", decode_bytes(w5, t5), med, mn, w5.G)
     del rows5
     med, mn = time_launches(lambda: ap.approxifer_locate_decode(p5, Yt, mt, Yh), 3, 10)
     entry("configs[4] locate + decode from trusted through approxifer_locate_decode (two launches at this size)",

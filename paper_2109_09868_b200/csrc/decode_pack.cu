@@ -203,6 +203,10 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
   // whole 16-byte columns and the last two floats go by hand.  Worker-major (WM; called by the whole warp): lane 0
   // announces the bytes, lane i starts the copy of worker i's rows of the item's groups, which land worker by
   // worker, GW rows apart; a last item whose pieces are not whole 16-byte columns goes by hand.
+  // (worker-major: where this lane's worker's batch starts, looked up once -- a per-lane index into the offset
+  // table in the parameter bank is a serialised load)
+  const float* my_batch = a.Yt;
+  if constexpr (WM) my_batch += a.rows.on ? a.rows.off[lane < W ? lane : 0] : (int64_t)lane * a.y_rs;
   auto issue = [&](int64_t g0, int slot) {
     const int ng = (int)min((int64_t)GW, a.G - g0);
     unsigned char* dst = slots + (size_t)slot * plan.in_bytes;
@@ -226,7 +230,7 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     } else {
       const uint32_t piece = (uint32_t)ng * plan.row_bytes;  // one worker's rows of the item's groups
       const bool whole = (piece & 15u) == 0;
-      const float* src = a.Yt + (a.rows.on ? a.rows.off[lane < W ? lane : 0] : (int64_t)lane * a.y_rs) + g0 * (int64_t)C;
+      const float* src = my_batch + g0 * (int64_t)C;
       unsigned char* mine_dst = dst + (uint32_t)lane * plan.y_row_step;
       if (!whole && lane < W)
         for (uint32_t f = 0; f < piece / 4u; ++f) reinterpret_cast<float*>(mine_dst)[f] = src[f];
