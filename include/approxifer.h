@@ -235,9 +235,11 @@ int approxifer_locate_decode(const approxifer_params* params, int64_t G, int64_t
  * its row of group g at element offset g * gstride (gstride >= D or C).  The pointers must be whole elements apart;
  * 16-byte aligned buffers with D (or C) and the strides multiples of 4 take the 128-bit path.  The encoder computes
  * every coded row once and stores each to its worker's buffer; the decoder and the locator read each present
- * worker's row from its buffer (the decoder with its per-column kernel).  Only plain global loads and stores
- * touch these buffers (no bulk asynchronous copies), so peer memory needs nothing but peer access enabled by the
- * caller.  Formulas, masks, outputs, status bits and return codes as in approxifer_encode / _decode / _locate;
+ * worker's row from its buffer.  The encoder, the locator and the decoder's per-column kernel touch these buffers
+ * with plain global loads and stores only; the decoder's packed-groups kernel (dense batches of 6-10 classes, 32 MB
+ * of predictions or more) reads them with bulk asynchronous copies into the issuing CTA's own shared memory (one
+ * copy per worker and work item, never multicast across a cluster).  Peer memory needs nothing but peer access
+ * enabled by the caller.  Formulas, masks, outputs, status bits and return codes as in approxifer_encode / _decode / _locate;
  * APPROXIFER_E_NULL also if one of the W pointers is NULL or not a whole number of elements from the first.
  */
 int approxifer_encode_scatter(const approxifer_params* params, int64_t G, int64_t D,
