@@ -238,7 +238,7 @@ int approxifer_locate_decode(const approxifer_params* params, int64_t G, int64_t
  * worker's row from its buffer.  The encoder, the locator and the decoder's per-column kernel touch these buffers
  * with plain global loads and stores only; the decoder's packed-groups kernel (dense batches of 6-10 classes, 32 MB
  * of predictions or more) reads them with bulk asynchronous copies into the issuing CTA's own shared memory (one
- * copy per worker and work item, never multicast across a cluster).  Peer memory needs nothing but peer access
+ * copy per worker and work item, each into one CTA's memory only).  Peer memory needs nothing but peer access
  * enabled by the caller.  Formulas, masks, outputs, status bits and return codes as in approxifer_encode / _decode / _locate;
  * APPROXIFER_E_NULL also if one of the W pointers is NULL or not a whole number of elements from the first.
  */
