@@ -140,7 +140,7 @@ __device__ __forceinline__ float p_hi(uint64_t v) { return __uint_as_float((uint
 // wtab[sg][i][j] = (w, w) with w = (-1)^sg / (alpha_j - beta_i): the signed weight, already duplicated for the
 // packed multiply-add (the sign flip is exact, so (s rg) y rounds like rg (s y)).
 // SIMPLE: one lane owns all the words of its rows (nch == 1, NW == C/2), so every offset is a compile-time constant.
-template <int NW, bool SIMPLE, bool ROT, bool WM>
+template <int NW, bool SIMPLE, bool ROT, bool WM, bool DEEP>
 __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
     decode_pack_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ DecodeTables tab,
                        const __grid_constant__ PackPlan plan) {
@@ -290,13 +290,12 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
       uint32_t r = 0;  // present workers so far = rank of the next one
       const unsigned char* yr = yg;
       const unsigned char* wr = wrow0;
-#pragma unroll 2
-      for (int i = 0; i < W; ++i, yr += plan.y_row_step, wr += plan.wrow_bytes) {
+      // one worker's row (an absent worker's row may be loaded; it is only used under `present`)
+      auto row = [&](int i) {
         uint64_t y[NW];
 #pragma unroll
-        for (int u = 0; u < NW; ++u) {  // (an absent worker's row may be loaded; it is only used under `present`)
+        for (int u = 0; u < NW; ++u)
           y[u] = (exact || u * nch + ch < Cw) ? *reinterpret_cast<const uint64_t*>(yr + woff(u)) : 0ull;
-        }
         if ((mask >> i) & 1u) {
           // the signed, duplicated weights of this lane's two queries
           const uint32_t odd = (literal ? (uint32_t)i : r) & 1u;
@@ -310,6 +309,17 @@ __global__ void __launch_bounds__(pack_max_warps(NW) * 32, 1)
           }
           ++r;
         }
+        yr += plan.y_row_step, wr += plan.wrow_bytes;
+      };
+      // (DEEP: unrolled by four where a group has three or more lanes, K >= 5: measured 1.00-1.14x there, 0.93x
+      // with one or two lanes per group; a kernel of its own, since the two loops side by side cost the shapes
+      // that take the short one 6-10 %)
+      if constexpr (DEEP) {
+#pragma unroll 4
+        for (int i = 0; i < W; ++i) row(i);
+      } else {
+#pragma unroll 2
+        for (int i = 0; i < W; ++i) row(i);
       }
       n = (int)r;
       // alpha_j == beta_i for a present worker i: the interpolant takes that worker's value
@@ -569,7 +579,7 @@ bool plan_pack(const DecodeArgs& a, int smem_per_sm, PackChoice* out) {
   return true;
 }
 
-template <int NW, bool SIMPLE, bool ROT, bool WM>
+template <int NW, bool SIMPLE, bool ROT, bool WM, bool DEEP>
 cudaError_t launch_pack(const DecodeArgs& a, const DecodeTables& tab, const PackChoice& c, const DeviceInfo& di,
                         cudaStream_t stream) {
   PackPlan plan;
@@ -590,12 +600,12 @@ cudaError_t launch_pack(const DecodeArgs& a, const DecodeTables& tab, const Pack
   plan.probe = a.tune.wait_limit != 0;
   plan.wait_limit = plan.probe ? a.tune.wait_limit : kPackWaitLimit;
   struct Tag {};
-  cudaError_t e = ensure_dynamic_smem<Tag>(decode_pack_kernel<NW, SIMPLE, ROT, WM>, di.ordinal, c.smem);
+  cudaError_t e = ensure_dynamic_smem<Tag>(decode_pack_kernel<NW, SIMPLE, ROT, WM, DEEP>, di.ordinal, c.smem);
   if (e != cudaSuccess) return e;
   int64_t grid = di.sms;
   const int64_t need = (plan.n_items + c.warps - 1) / c.warps;
   if (grid > need) grid = need;
-  decode_pack_kernel<NW, SIMPLE, ROT, WM><<<(unsigned)grid, c.warps * 32, c.smem, stream>>>(a, tab, plan);
+  decode_pack_kernel<NW, SIMPLE, ROT, WM, DEEP><<<(unsigned)grid, c.warps * 32, c.smem, stream>>>(a, tab, plan);
   count_launch();
   return cudaGetLastError();
 }
@@ -607,13 +617,22 @@ cudaError_t dispatch_nw(const DecodeArgs& a, const DecodeTables& tab, const Pack
     return cudaErrorInvalidValue;
   } else {
     if (c.nw == NW) {
+      const bool deep = c.jt >= 3;  // K >= 5
       if (c.nch == 1 && NW * 2 == a.C) {
-        if (c.worker_major) return launch_pack<NW, true, false, true>(a, tab, c, di, stream);
-        if (c.rot_groups != 0) return launch_pack<NW, true, true, false>(a, tab, c, di, stream);
-        return launch_pack<NW, true, false, false>(a, tab, c, di, stream);
+        if (c.worker_major)
+          return deep ? launch_pack<NW, true, false, true, true>(a, tab, c, di, stream)
+                      : launch_pack<NW, true, false, true, false>(a, tab, c, di, stream);
+        if (c.rot_groups != 0)
+          return deep ? launch_pack<NW, true, true, false, true>(a, tab, c, di, stream)
+                      : launch_pack<NW, true, true, false, false>(a, tab, c, di, stream);
+        return deep ? launch_pack<NW, true, false, false, true>(a, tab, c, di, stream)
+                    : launch_pack<NW, true, false, false, false>(a, tab, c, di, stream);
       }
-      if (c.worker_major) return launch_pack<NW, false, false, true>(a, tab, c, di, stream);
-      return launch_pack<NW, false, false, false>(a, tab, c, di, stream);
+      if (c.worker_major)
+        return deep ? launch_pack<NW, false, false, true, true>(a, tab, c, di, stream)
+                    : launch_pack<NW, false, false, true, false>(a, tab, c, di, stream);
+      return deep ? launch_pack<NW, false, false, false, true>(a, tab, c, di, stream)
+                  : launch_pack<NW, false, false, false, false>(a, tab, c, di, stream);
     }
     return dispatch_nw<NW + 1>(a, tab, c, di, stream);
   }
