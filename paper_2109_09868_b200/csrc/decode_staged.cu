@@ -11,7 +11,7 @@
 //
 // A work item is (group, tile of COLS 16-byte columns).  SPLIT*COLS compute threads work on it:
 // thread = (thread group h, column); group h forms the queries j = h*KT .. h*KT+KT-1 (KT = ceil(K/SPLIT)).
-// With SPLIT = 1 (the default where it fits: K <= 8 or 13 .. 16, COLS = 256, one CTA per SM) every payload word is read
+// With SPLIT = 1 (the default where it fits: K <= 16, COLS = 256, one CTA per SM; K = 9 .. 12 on 16,384 groups or more take SPLIT = 2) every payload word is read
 // from shared memory once and a thread keeps all K accumulators per payload element; with SPLIT = 2 or 4 the
 // thread groups share each column's payload, every thread keeps only KT accumulators, and there are more warps
 // per byte of ring (two CTAs per SM).  The FMAs are packed (fma.rn.f32x2: the weights of two adjacent
@@ -525,7 +525,9 @@ cudaError_t dispatch_whole(const DecodeArgs& a, const DecodeTables& tab, cudaStr
       // (K = 9 .. 12: two thread groups of up to 6 queries on the same 256-column items measured 1.07-1.09x
       // this plan on 3 GB problems, K = 10, 12, C = 1000, 2000; equal at K = 8, 1.01x at K = 16, where the single
       // group sustains better under the power cap)
-      const bool two_groups_better = a.K >= 9 && a.K <= 12;
+      // ... and only from 16,384 groups on: on 4,096 groups (28 items per CTA, run right after the encoder under
+      // the power cap) the single group measured 2-5 % faster.
+      const bool two_groups_better = a.K >= 9 && a.K <= 12 && a.G >= 16384;
       const bool want = a.tune.split == 1 || (a.tune.split == 0 && (a.tune.cols == 0 || a.tune.cols == 256) &&
                                               waste256 <= waste128 && !two_groups_better);
       *taken = (want || a.bf16) && fits_256<KT, 1>(a);
